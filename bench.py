@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the WindowKV prefill-compression hot path (score -> pool -> top-k -> gather).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C3]
+
+One step = one `wkv_compress_group` call on one layer group of the workload
+(leader scoring + selection, then the shared-index gather of all gamma layers),
+rotating over the model's groups so that every step reads cold HBM.  Prints one
+JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_17922_b200 import workloads as wl   # noqa: E402
+
+METRIC = "prefill-compression tokens/s per layer group"
+UNIT = "tokens/s"
+
+
+def pick_workload(name: str):
+    if name == "C2":
+        return wl.llama8b_single_group(wl.TASK_AGGREGATION)
+    if name == "C4":
+        return wl.mistral_needle(32768, 0.5)
+    return wl.ALL_CONFIGS[name]()
+
+
+def algorithmic_bytes(w, prob) -> dict:
+    """Bytes the method must move for one group (leader K once, Q_obs, and read+write of the
+    retained rows of K and V of every layer) with the per-stage split."""
+    e = 4 if w.dtype == "f32" else 2
+    tokens = int(w.seqlens().sum())
+    score = tokens * w.n_kv_heads * w.head_dim * e + w.batch * w.n_q_heads * w.l_obs * w.head_dim * e
+    keep_rows = 0
+    for n, b in zip(w.seqlens(), w.budgets()):
+        k = min(max(0, (int(b) - w.l_obs) // w.window), -(-max(int(n) - w.l_obs, 0) // w.window))
+        keep_rows += k * w.window + min(w.l_obs, int(n))
+    gather = w.gamma * 2 * 2 * keep_rows * w.n_kv_heads * w.head_dim * e
+    return {"score": score, "gather": gather, "total": score + gather, "tokens": tokens}
+
+
+def peaks() -> dict:
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def ncu_traffic(kernel: str):
+    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(p):
+        return json.load(open(p)).get(kernel)
+    return None
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle_groups(w, groups, min_seconds: float, max_groups: int):
+    """Runs the CPU oracle on whole groups until `min_seconds` of work; returns (tokens/s, n_groups, s)."""
+    import oracle
+    tokens = int(w.seqlens().sum())
+    done, spent = 0, 0.0
+    while (spent < min_seconds and done < max_groups) or done == 0:
+        grp = groups[done % len(groups)]
+        t0 = time.perf_counter()
+        oracle.compress_group(grp["q_obs"], grp["k_layers"], grp["v_layers"], n_kv_heads=w.n_kv_heads,
+                              l_obs=w.l_obs, window=w.window, task=w.task, top_p=w.top_p,
+                              max_seqlen=w.max_seqlen, budgets=grp["budgets"], cu_seqlens=grp["cu_seqlens"])
+        spent += time.perf_counter() - t0
+        done += 1
+    return tokens * done / spent, done, spent
+
+
+def run_reference(args) -> None:
+    """The reference arm: the CPU oracle, as it stands, on the same workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    w = pick_workload(args.workload)
+    n_distinct = min(w.n_groups, 2)
+    groups = [wl.make_group(w, g) for g in range(n_distinct)]
+    tokens = int(w.seqlens().sum())
+
+    def step(i):
+        grp = groups[i % n_distinct]
+        oracle.compress_group(grp["q_obs"], grp["k_layers"], grp["v_layers"], n_kv_heads=w.n_kv_heads,
+                              l_obs=w.l_obs, window=w.window, task=w.task, top_p=w.top_p,
+                              max_seqlen=w.max_seqlen, budgets=grp["budgets"], cu_seqlens=grp["cu_seqlens"])
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(i)
+    dt = time.perf_counter() - t0
+    value = tokens * args.steps / dt
+    cores = oracle.num_threads()
+    sample = f"one whole layer group ({w.gamma} layers, {tokens} tokens) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+        "data": "synthetic (seeded; shapes of the paper's long-context workloads)",
+        "config": {"workload": w.name, "batch": w.batch, "seq_len": w.max_seqlen, "layers_per_group": w.gamma},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=48)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
+    ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05"])
+    ap.add_argument("--groups", type=int, default=0, help="distinct groups kept on the device (0 = all)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_17922_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()          # fails loudly if the CUDA library is missing
+
+    w = pick_workload(args.workload)
+    impl = {"auto": binding.WKV_SCORE_AUTO, "simt": binding.WKV_SCORE_SIMT,
+            "tcgen05": binding.WKV_SCORE_TCGEN05}[args.score_impl]
+    prob = binding.Problem.from_workload(w, score_impl=impl)
+    alg = algorithmic_bytes(w, prob)
+    tokens = alg["tokens"]
+
+    # ---- inputs: every group of the model resident in HBM (each rank its own copy: weak scaling)
+    n_groups = w.n_groups if args.groups <= 0 else min(args.groups, w.n_groups)
+    host_groups, dev_groups = [], []
+    for g in range(n_groups):
+        grp = wl.make_group(w, g)
+        if g < 2:
+            host_groups.append(grp)
+        dev_groups.append({"q": binding.to_device(grp["q_obs"]),
+                           "k": [binding.to_device(x) for x in grp["k_layers"]],
+                           "v": [binding.to_device(x) for x in grp["v_layers"]]})
+    out = prob.alloc_outputs(w.gamma)
+    work = prob.alloc_workspace()
+    stream = torch.cuda.current_stream()
+    resident = sum(t.numel() * t.element_size() for d in dev_groups for t in d["k"] + d["v"])
+    flush = None
+    if resident < 512 * 1024 * 1024:       # small workloads fit L2: flush between steps
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def step(i: int) -> None:
+        d = dev_groups[i % n_groups]
+        if flush is not None:
+            flush.fill_(i & 0xFF)
+        binding.wkv_compress_group(prob, d["q"], d["k"], d["v"], out["k_out"], out["v_out"],
+                                   out["window_scores"], out["window_idx"], out["kept_len"], work,
+                                   keep_capacity=out["keep_capacity"], stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.wkv_launch_count()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+    else:                                   # time each step alone so that the flush is not counted
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for i in range(args.steps):
+            d = dev_groups[i % n_groups]
+            flush.fill_(i & 0xFF)
+            evs[i][0].record(stream)
+            binding.wkv_compress_group(prob, d["q"], d["k"], d["v"], out["k_out"], out["v_out"],
+                                       out["window_scores"], out["window_idx"], out["kept_len"], work,
+                                       keep_capacity=out["keep_capacity"], stream=stream)
+            evs[i][1].record(stream)
+        barrier()
+        ms_total = sum(a.elapsed_time(b) for a, b in evs)
+    launches = binding.wkv_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = tokens * world / (ms_per_step * 1e-3)
+
+    # ---- per-stage device times (CUDA events on the launching stream, same rotation)
+    def time_stage(fn, reps: int) -> float:
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        tot = 0.0
+        pairs = []
+        for i in range(reps):
+            if flush is not None:
+                flush.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(i)
+            b.record(stream)
+            pairs.append((a, b))
+        torch.cuda.synchronize()
+        tot = sum(a.elapsed_time(b) for a, b in pairs)
+        return tot / reps
+
+    reps = max(16, min(args.steps, 64))
+    ms_score = time_stage(lambda i: binding.wkv_score_windows(
+        prob, dev_groups[i % n_groups]["q"], dev_groups[i % n_groups]["k"][0], out["window_scores"], None, work,
+        stream=stream), reps)
+    ms_select = time_stage(lambda i: binding.wkv_select_topk_windows(
+        prob, out["window_scores"], out["window_idx"], out["kept_len"], stream=stream), reps)
+    ms_gather = time_stage(lambda i: binding.wkv_gather_kv(
+        prob, dev_groups[i % n_groups]["k"], dev_groups[i % n_groups]["v"], out["window_idx"], out["k_out"],
+        out["v_out"], keep_capacity=out["keep_capacity"], stream=stream), reps)
+
+    pk = peaks()
+    dominant = "gather" if ms_gather >= ms_score else "score"
+    dom_ms = ms_gather if dominant == "gather" else ms_score
+    achieved = alg[dominant] / (dom_ms * 1e-3) / 1e9
+    kernel_name = "gather_kv_kernel" if dominant == "gather" else "score kernels (stats + score/pool)"
+    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": pk["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
+                "traffic": ncu_traffic(dominant), "algorithmic_bytes_per_launch": alg[dominant]}
+    path_frac = alg["total"] / (ms_per_step * 1e-3) / 1e9 / pk["hbm_gbs"]
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda a: binding.to_device(a, "cpu").pin_memory()
+        hsets = []
+        for grp in host_groups:
+            hsets.append({"q": pin(grp["q_obs"]), "k": [pin(x) for x in grp["k_layers"]],
+                          "v": [pin(x) for x in grp["v_layers"]]})
+        h_k_out = [torch.empty_like(t, device="cpu").pin_memory() for t in out["k_out"]]
+        h_v_out = [torch.empty_like(t, device="cpu").pin_memory() for t in out["v_out"]]
+        h_idx = torch.empty_like(out["window_idx"], device="cpu").pin_memory()
+        h_kept = torch.empty_like(out["kept_len"], device="cpu").pin_memory()
+        stage = dev_groups[0]
+
+        def e2e_step(i):
+            hs = hsets[i % len(hsets)]
+            binding.wkv_compress_group_host(prob, hs["q"], hs["k"], hs["v"], h_k_out, h_v_out, h_idx, h_kept,
+                                            stage["q"], stage["k"], stage["v"], out["k_out"], out["v_out"],
+                                            out["window_idx"], out["kept_len"], out["keep_capacity"], work,
+                                            stream=stream)
+        e2e_steps = max(3, min(args.steps, 12))
+        for i in range(2):
+            e2e_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        barrier()
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        nb = lambda t: t.numel() * t.element_size()
+        h2d = nb(hsets[0]["q"]) + sum(nb(x) for x in hsets[0]["k"] + hsets[0]["v"])
+        d2h = sum(nb(x) for x in h_k_out + h_v_out) + nb(h_idx) + nb(h_kept)
+        e2e = {"value": tokens * world * e2e_steps / float(tt.item()), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    # ---- the oracle on the host cores (rank 0, single-GPU runs only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        v, n_done, spent = time_oracle_groups(w, host_groups, 10.0, 24)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"{n_done} whole layer groups of {w.name} ({spent:.1f} s)"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "accum_dtype": "f32",
+            "data": "synthetic (seeded; shapes of the paper's long-context workloads)",
+            "config": {"workload": w.name, "batch": w.batch, "seq_len": w.max_seqlen, "layers_per_group": w.gamma,
+                       "groups_rotated": n_groups, "l_obs": w.l_obs, "window": w.window,
+                       "budget_tokens": int(w.budgets()[0]), "score_impl": args.score_impl,
+                       "cold_cache": "flush of 256 MB between steps" if flush is not None
+                       else f"{n_groups} groups rotated ({resident / 1e9:.2f} GB resident, larger than L2)"},
+            "gpu_launches": int(launches),
+            "path_hbm_frac": path_frac,
+            "path_algorithmic_bytes": alg["total"],
+            "stages_ms": {"score": ms_score, "select": ms_select, "gather": ms_gather},
+            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "clocks": clocks,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,195 @@
+/*
+ * wkv — WindowKV prefill-time KV-cache window selection for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  Notation follows the paper (section 2.2.1 / 2.2.2):
+ *   n      context length of a sequence (observation window included)
+ *   alpha  observation-window length   (field l_obs)
+ *   omega  review-window length        (field window)
+ *   p      Top-p count of Eq. 4        (field top_p, aggregation task only)
+ *   gamma  layers per group            (argument n_layers)
+ *   b      per-layer KV budget in tokens, observation window included
+ *   G      query heads per KV head = n_q_heads / n_kv_heads
+ * A "unit" is one (sequence, KV head) pair.  Derived integers, identical on
+ * host and device:
+ *   K_w = ceil((n - alpha)/omega)  (0 when n <= alpha)          — Eq. 3
+ *   k   = min(K_w, max(0, floor((b - alpha)/omega)))            — budget sentence after Eq. 4
+ *
+ * General conventions
+ *   - Every pointer marked DEVICE is device memory owned by the caller; HOST
+ *     pointers are ordinary host memory read before the function returns.
+ *     The library allocates and frees nothing and keeps no state between
+ *     calls other than a launch counter.
+ *   - All device work is enqueued on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and the functions return
+ *     without synchronising.
+ *   - Argument errors are detected on the host before anything is enqueued
+ *     and returned as a wkv_status (0 = success).  wkv_last_error_detail()
+ *     gives a thread-local human-readable reason for the last failure.
+ *   - Tensors have the head dimension contiguous.  K/V element (b, h, j, c)
+ *     lives at  base[(off_b + j)*stride_t + b*stride_b + h*stride_h + c]
+ *     where off_b = cu_seqlens[b] for the packed layout (then stride_b = 0)
+ *     and 0 for the dense layout.  Dense [B,H_kv,N,d]:
+ *     stride_b = H_kv*N*d, stride_h = N*d, stride_t = d.  Packed [T,H_kv,d]:
+ *     stride_b = 0, stride_h = d, stride_t = H_kv*d.
+ *     Q_obs element (b, hq, i, c) at q[b*q_stride_b + hq*q_stride_h + i*q_stride_t + c],
+ *     i = 0..alpha-1 being positions n-alpha .. n-1 of the sequence.
+ *   - Base pointers and row strides must be 16-byte aligned.
+ */
+#ifndef WKV_H_
+#define WKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WKV_OK = 0,
+    WKV_ERR_NULL = 1,        /* a required pointer is NULL */
+    WKV_ERR_SHAPE = 2,       /* inconsistent or non-positive sizes */
+    WKV_ERR_DTYPE = 3,
+    WKV_ERR_BUDGET = 4,      /* negative budget */
+    WKV_ERR_WORKSPACE = 5,   /* workspace missing, too small or misaligned */
+    WKV_ERR_ALIGN = 6,       /* pointer or stride not 16-byte aligned */
+    WKV_ERR_UNSUPPORTED = 7, /* shape outside what the kernels cover */
+    WKV_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed */
+    WKV_ERR_LIMIT = 9        /* size beyond a documented fixed maximum */
+} wkv_status;
+
+typedef enum { WKV_F32 = 0, WKV_BF16 = 1 } wkv_dtype;
+typedef enum { WKV_TASK_LOCALIZATION = 0, WKV_TASK_AGGREGATION = 1 } wkv_task;
+/* which score kernel family to use: AUTO picks the tensor-core (tcgen05) kernels
+ * for bf16 inputs with head_dim 64 or 128 and G*alpha <= 256, else the plain
+ * CUDA-core kernels. */
+typedef enum { WKV_SCORE_AUTO = 0, WKV_SCORE_SIMT = 1, WKV_SCORE_TCGEN05 = 2 } wkv_score_impl;
+
+#define WKV_MAX_GROUP_LAYERS 32
+
+typedef struct {
+    uint32_t struct_size;   /* sizeof(wkv_shape), checked */
+    int32_t dtype;          /* wkv_dtype of Q, K, V and of the compact cache */
+    int32_t batch;          /* B */
+    int32_t n_q_heads;      /* H_q, a multiple of n_kv_heads */
+    int32_t n_kv_heads;     /* H_kv */
+    int32_t head_dim;       /* d, a multiple of 8 (bf16) / 4 (fp32) */
+    int32_t l_obs;          /* alpha >= 1 */
+    int32_t window;         /* omega >= 1 */
+    int32_t top_p;          /* p for WKV_TASK_AGGREGATION; 0 => ceil(omega/2) */
+    int32_t task;           /* wkv_task: selects p = omega (localization) or p = top_p */
+    int32_t max_seqlen;     /* N: the common length (dense) or an upper bound (packed) */
+    int32_t budget;         /* per-layer budget b for every sequence, used when budgets_host == NULL */
+    int32_t score_impl;     /* wkv_score_impl */
+    int32_t reserved;       /* must be 0 */
+    const int32_t *cu_seqlens_host; /* HOST  [B+1] or NULL => dense, every n_b = max_seqlen */
+    const int32_t *cu_seqlens_dev;  /* DEVICE copy of the same array (required iff the host one is given) */
+    const int32_t *budgets_host;    /* HOST  [B] per-sequence budgets, or NULL => `budget` */
+    const int32_t *budgets_dev;     /* DEVICE copy of the same array (required iff the host one is given) */
+    int64_t stride_b, stride_h, stride_t;       /* K/V element strides */
+    int64_t q_stride_b, q_stride_h, q_stride_t; /* Q_obs element strides */
+} wkv_shape;
+
+/* ---- host-side integer helpers (Eq. 3 and the budget sentence after Eq. 4) ---- */
+int32_t wkv_num_windows(int32_t n, int32_t alpha, int32_t omega);                   /* K_w */
+int32_t wkv_num_selected(int32_t n, int32_t alpha, int32_t omega, int32_t budget);  /* k   */
+/* Leading sizes of the output arrays for a whole batch: */
+int32_t wkv_kw_max(const wkv_shape *s);   /* max_b K_w,b, at least 1 */
+int32_t wkv_k_max(const wkv_shape *s);    /* max_b k_b,   at least 1 */
+int32_t wkv_keep_max(const wkv_shape *s); /* max_b (k_b*omega + min(alpha, n_b)): row capacity of the dense compact cache */
+
+/* Bytes of DEVICE scratch that wkv_score_windows / wkv_compress_group need for this
+ * shape (256-byte aligned base expected).  Returns 0 for an invalid shape. */
+size_t wkv_workspace_bytes(const wkv_shape *s);
+
+/*
+ * Eq. 1-4 for the group's leader layer.
+ * For every unit: logits of the G*alpha observation rows against every key the row
+ * may attend to (causal: keys 0..position), softmax per row (Eq. 1), sum over the
+ * rows and the G heads for each review token j < n - alpha (Eq. 2), then the
+ * window score s_k = sum(Top-p of window k)/min(p, |window k|) (Eq. 3-4; the last
+ * window may be shorter than omega).  fp32 accumulation throughout.
+ *   q_obs          DEVICE  observation queries of the leader
+ *   k_leader       DEVICE  keys of the leader
+ *   window_scores  DEVICE  out, float [B, H_kv, wkv_kw_max()] ; entries >= K_w,b are not written
+ *   token_scores   DEVICE  out or NULL, float [B, H_kv, max(1, max_seqlen - alpha)] ; t_j of Eq. 2
+ *   workspace      DEVICE  scratch of wkv_workspace_bytes() bytes
+ */
+int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader,
+                      float *window_scores, float *token_scores,
+                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Budgeted selection (sentence after Eq. 4): per unit the k highest window scores,
+ * ties to the lower window index, indices written in ascending order.
+ *   window_scores  DEVICE  in,  float [B, H_kv, wkv_kw_max()]
+ *   window_idx     DEVICE  out, int32 [B, H_kv, wkv_k_max()], entries >= k_b set to -1
+ *   kept_len       DEVICE  out, int32 [B, H_kv]: rows of the compact cache of the unit
+ *                  (tokens in the selected windows + min(alpha, n_b))
+ */
+int wkv_select_topk_windows(const wkv_shape *s, const float *window_scores,
+                            int32_t *window_idx, int32_t *kept_len, void *cuda_stream);
+
+/*
+ * Intra-group index sharing (section 2.2.2): builds the compact cache of n_layers
+ * layers from one set of window indices.  Output row r of a unit is source row
+ * idx[r/omega]*omega + r%omega for the retained review rows (ascending position),
+ * followed by the observation rows n-alpha .. n-1.  Bit copies.
+ *   k_layers, v_layers          HOST arrays [n_layers] of DEVICE pointers (inputs, layout of `s`)
+ *   k_out_layers, v_out_layers  HOST arrays [n_layers] of DEVICE pointers (outputs)
+ *   window_idx                  DEVICE int32 [B, H_kv, wkv_k_max()] as written by the selection
+ *   cu_seqlens_out              DEVICE int32 [B+1] or NULL.
+ *       NULL  => dense output [B, H_kv, keep_capacity, d]; rows >= kept_len are not written.
+ *       else  => packed output [T_out, H_kv, d], sequence b starting at row cu_seqlens_out[b].
+ *   keep_capacity               rows per unit of the dense output (>= wkv_keep_max()); ignored when packed
+ * Either of v_layers / v_out_layers may be NULL to gather keys only.
+ */
+int wkv_gather_kv(const wkv_shape *s, int32_t n_layers,
+                  const void *const *k_layers, const void *const *v_layers,
+                  const int32_t *window_idx,
+                  void *const *k_out_layers, void *const *v_out_layers,
+                  const int32_t *cu_seqlens_out, int32_t keep_capacity, void *cuda_stream);
+
+/*
+ * One layer group (sections 2.2.1-2.2.2): score + select on k_layers[0] with q_obs_leader,
+ * then the shared-index gather of all n_layers layers.  Arguments as above;
+ * window_scores may be NULL (then the scores live in the workspace only).
+ */
+int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
+                       const void *const *k_layers, const void *const *v_layers,
+                       void *const *k_out_layers, void *const *v_out_layers,
+                       float *window_scores, int32_t *window_idx, int32_t *kept_len,
+                       const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The same group with every tensor in HOST memory (pinned memory recommended): the
+ * inputs are copied to caller-provided DEVICE staging buffers, the group is
+ * compressed there, and indices, kept lengths and the compact caches are copied
+ * back; the function returns after the stream has been synchronised.
+ *   *_host arguments    HOST pointers / HOST arrays of HOST pointers
+ *   *_dev arguments     DEVICE staging of the same sizes (HOST arrays of DEVICE pointers)
+ *   bytes_per_layer     size of one K (or V) tensor; out_bytes_per_layer of one compact cache
+ * Dense output layout only.
+ */
+int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers,
+                            const void *q_obs_host, size_t q_bytes,
+                            const void *const *k_layers_host, const void *const *v_layers_host,
+                            size_t bytes_per_layer,
+                            void *const *k_out_layers_host, void *const *v_out_layers_host,
+                            size_t out_bytes_per_layer,
+                            int32_t *window_idx_host, int32_t *kept_len_host,
+                            void *q_obs_dev, void *const *k_layers_dev, void *const *v_layers_dev,
+                            void *const *k_out_layers_dev, void *const *v_out_layers_dev,
+                            int32_t *window_idx_dev, int32_t *kept_len_dev, int32_t keep_capacity,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+const char *wkv_status_string(int status);
+const char *wkv_last_error_detail(void);
+/* Number of kernels the library has launched from this process (all threads). */
+uint64_t wkv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WKV_H_ */

@@ -1,0 +1,298 @@
+"""Thin ctypes binding of the C-ABI library (include/wkv.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  Tensors are torch CUDA tensors used purely as device memory; their
+`data_ptr()` and the current stream's handle are what crosses the boundary.
+There is no CPU fallback: if the shared library is missing, loading fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libwkv.so")
+
+WKV_F32, WKV_BF16 = 0, 1
+WKV_TASK_LOCALIZATION, WKV_TASK_AGGREGATION = 0, 1
+WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05 = 0, 1, 2
+WKV_MAX_GROUP_LAYERS = 32
+
+EXPORTED_SYMBOLS = [
+    "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max",
+    "wkv_workspace_bytes", "wkv_score_windows", "wkv_select_topk_windows", "wkv_gather_kv",
+    "wkv_compress_group", "wkv_compress_group_host", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_launch_count",
+]
+
+
+class WkvShape(ctypes.Structure):
+    """Mirror of `wkv_shape`."""
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("dtype", ctypes.c_int32),
+        ("batch", ctypes.c_int32),
+        ("n_q_heads", ctypes.c_int32),
+        ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("l_obs", ctypes.c_int32),
+        ("window", ctypes.c_int32),
+        ("top_p", ctypes.c_int32),
+        ("task", ctypes.c_int32),
+        ("max_seqlen", ctypes.c_int32),
+        ("budget", ctypes.c_int32),
+        ("score_impl", ctypes.c_int32),
+        ("reserved", ctypes.c_int32),
+        ("cu_seqlens_host", ctypes.c_void_p),
+        ("cu_seqlens_dev", ctypes.c_void_p),
+        ("budgets_host", ctypes.c_void_p),
+        ("budgets_dev", ctypes.c_void_p),
+        ("stride_b", ctypes.c_int64),
+        ("stride_h", ctypes.c_int64),
+        ("stride_t", ctypes.c_int64),
+        ("q_stride_b", ctypes.c_int64),
+        ("q_stride_h", ctypes.c_int64),
+        ("q_stride_t", ctypes.c_int64),
+    ]
+
+
+class WkvError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str):
+        super().__init__(f"{what}: status {status} ({detail})")
+        self.status = status
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libwkv.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_17922_b200.build` "
+                           "(needs nvcc); this package has no other implementation of the path")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    sp = ctypes.POINTER(WkvShape)
+    L.wkv_num_windows.restype = i32
+    L.wkv_num_windows.argtypes = [i32, i32, i32]
+    L.wkv_num_selected.restype = i32
+    L.wkv_num_selected.argtypes = [i32, i32, i32, i32]
+    for name in ("wkv_kw_max", "wkv_k_max", "wkv_keep_max"):
+        getattr(L, name).restype = i32
+        getattr(L, name).argtypes = [sp]
+    L.wkv_workspace_bytes.restype = sz
+    L.wkv_workspace_bytes.argtypes = [sp]
+    L.wkv_score_windows.restype = ctypes.c_int
+    L.wkv_score_windows.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp]
+    L.wkv_select_topk_windows.restype = ctypes.c_int
+    L.wkv_select_topk_windows.argtypes = [sp, vp, vp, vp, vp]
+    L.wkv_gather_kv.restype = ctypes.c_int
+    L.wkv_gather_kv.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
+    L.wkv_compress_group.restype = ctypes.c_int
+    L.wkv_compress_group.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.wkv_compress_group_host.restype = ctypes.c_int
+    L.wkv_compress_group_host.argtypes = [sp, i32, vp, sz, vp, vp, sz, vp, vp, sz, vp, vp,
+                                          vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.wkv_status_string.restype = ctypes.c_char_p
+    L.wkv_status_string.argtypes = [ctypes.c_int]
+    L.wkv_last_error_detail.restype = ctypes.c_char_p
+    L.wkv_last_error_detail.argtypes = []
+    L.wkv_launch_count.restype = ctypes.c_uint64
+    L.wkv_launch_count.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        L = lib()
+        raise WkvError(status, what, f"{L.wkv_status_string(status).decode()}: "
+                                     f"{L.wkv_last_error_detail().decode()}")
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _ptr_array(tensors: Optional[Sequence]) -> Optional[ctypes.Array]:
+    if tensors is None:
+        return None
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t)
+    return arr
+
+
+class Problem:
+    """A `wkv_shape` together with the host/device arrays it points to (kept alive here)."""
+
+    def __init__(self, *, dtype: str, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 l_obs: int, window: int, task: int, top_p: int, max_seqlen: int,
+                 budgets: Sequence[int], cu_seqlens: Optional[Sequence[int]] = None,
+                 kv_layout: str = "bhnd", score_impl: int = WKV_SCORE_AUTO, device=None):
+        import torch
+        self.dtype = dtype
+        self.elem_bytes = 4 if dtype == "f32" else 2
+        self.torch_dtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        self.device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        s = WkvShape()
+        s.struct_size = ctypes.sizeof(WkvShape)
+        s.dtype = WKV_F32 if dtype == "f32" else WKV_BF16
+        s.batch, s.n_q_heads, s.n_kv_heads, s.head_dim = batch, n_q_heads, n_kv_heads, head_dim
+        s.l_obs, s.window, s.top_p, s.task = l_obs, window, top_p, task
+        s.max_seqlen = max_seqlen
+        s.score_impl = score_impl
+        self.budgets_host = np.ascontiguousarray(budgets, dtype=np.int32)
+        assert len(self.budgets_host) == batch
+        self.budgets_dev = torch.from_numpy(self.budgets_host).to(self.device)
+        s.budget = int(self.budgets_host[0])
+        s.budgets_host = self.budgets_host.ctypes.data
+        s.budgets_dev = self.budgets_dev.data_ptr()
+        self.packed = cu_seqlens is not None
+        if self.packed:
+            self.cu_host = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+            self.cu_dev = torch.from_numpy(self.cu_host).to(self.device)
+            s.cu_seqlens_host = self.cu_host.ctypes.data
+            s.cu_seqlens_dev = self.cu_dev.data_ptr()
+            s.stride_b, s.stride_h, s.stride_t = 0, head_dim, n_kv_heads * head_dim
+            self.seqlens = np.diff(self.cu_host)
+        else:
+            self.cu_host = self.cu_dev = None
+            if kv_layout == "bhnd":
+                s.stride_b, s.stride_h, s.stride_t = n_kv_heads * max_seqlen * head_dim, max_seqlen * head_dim, head_dim
+            elif kv_layout == "bnhd":
+                s.stride_b, s.stride_h, s.stride_t = max_seqlen * n_kv_heads * head_dim, head_dim, n_kv_heads * head_dim
+            else:
+                raise ValueError(kv_layout)
+            self.seqlens = np.full(batch, max_seqlen, dtype=np.int32)
+        s.q_stride_b, s.q_stride_h, s.q_stride_t = n_q_heads * l_obs * head_dim, l_obs * head_dim, head_dim
+        self.shape = s
+        L = lib()
+        self.kw_max = L.wkv_kw_max(ctypes.byref(s))
+        self.k_max = L.wkv_k_max(ctypes.byref(s))
+        self.keep_max = L.wkv_keep_max(ctypes.byref(s))
+        self.workspace_bytes = L.wkv_workspace_bytes(ctypes.byref(s))
+        if self.kw_max == 0:
+            raise WkvError(-1, "wkv_shape", L.wkv_last_error_detail().decode())
+        self.units = batch * n_kv_heads
+        self.nr_max = max(1, max_seqlen - l_obs)
+
+    @classmethod
+    def from_workload(cls, w, score_impl: int = WKV_SCORE_AUTO, device=None) -> "Problem":
+        """Builds the shape of a `workloads.Workload`."""
+        return cls(dtype=w.dtype, batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                   head_dim=w.head_dim, l_obs=w.l_obs, window=w.window, task=w.task, top_p=w.top_p,
+                   max_seqlen=w.max_seqlen, budgets=w.budgets(),
+                   cu_seqlens=w.cu_seqlens() if w.ragged else None, score_impl=score_impl, device=device)
+
+    # ---- caller-side allocations (torch is the allocator, nothing else) ----
+    def alloc_workspace(self):
+        import torch
+        return torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+
+    def alloc_outputs(self, n_layers: int, fill_byte: Optional[int] = None, keep_capacity: Optional[int] = None):
+        import torch
+        cap = self.keep_max if keep_capacity is None else keep_capacity
+        B, H, d = self.shape.batch, self.shape.n_kv_heads, self.shape.head_dim
+
+        def mk():
+            t = torch.empty((B, H, cap, d), dtype=self.torch_dtype, device=self.device)
+            if fill_byte is not None:
+                t.view(torch.uint8).fill_(fill_byte)
+            return t
+        return {
+            "window_scores": torch.full((B, H, self.kw_max), float("nan"), dtype=torch.float32, device=self.device),
+            "window_idx": torch.full((B, H, self.k_max), -7, dtype=torch.int32, device=self.device),
+            "kept_len": torch.full((B, H), -7, dtype=torch.int32, device=self.device),
+            "k_out": [mk() for _ in range(n_layers)],
+            "v_out": [mk() for _ in range(n_layers)],
+            "keep_capacity": cap,
+        }
+
+
+def wkv_score_windows(prob: Problem, q_obs, k_leader, window_scores, token_scores, workspace, stream=None) -> None:
+    _check(lib().wkv_score_windows(ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader), _ptr(window_scores),
+                                   _ptr(token_scores), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "wkv_score_windows")
+
+
+def wkv_select_topk_windows(prob: Problem, window_scores, window_idx, kept_len, stream=None) -> None:
+    _check(lib().wkv_select_topk_windows(ctypes.byref(prob.shape), _ptr(window_scores), _ptr(window_idx),
+                                         _ptr(kept_len), _stream(stream)), "wkv_select_topk_windows")
+
+
+def wkv_gather_kv(prob: Problem, k_layers, v_layers, window_idx, k_out_layers, v_out_layers,
+                  cu_seqlens_out=None, keep_capacity: int = 0, stream=None) -> None:
+    _check(lib().wkv_gather_kv(ctypes.byref(prob.shape), len(k_layers), _ptr_array(k_layers),
+                               _ptr_array(v_layers), _ptr(window_idx), _ptr_array(k_out_layers),
+                               _ptr_array(v_out_layers), _ptr(cu_seqlens_out), keep_capacity, _stream(stream)),
+           "wkv_gather_kv")
+
+
+def wkv_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers,
+                       window_scores, window_idx, kept_len, workspace, cu_seqlens_out=None,
+                       keep_capacity: int = 0, stream=None) -> None:
+    _check(lib().wkv_compress_group(ctypes.byref(prob.shape), len(k_layers), _ptr(q_obs_leader),
+                                    _ptr_array(k_layers), _ptr_array(v_layers), _ptr_array(k_out_layers),
+                                    _ptr_array(v_out_layers), _ptr(window_scores), _ptr(window_idx),
+                                    _ptr(kept_len), _ptr(cu_seqlens_out), keep_capacity, _ptr(workspace),
+                                    workspace.numel(), _stream(stream)), "wkv_compress_group")
+
+
+def wkv_compress_group_host(prob: Problem, q_obs_host, k_layers_host, v_layers_host, k_out_host, v_out_host,
+                            window_idx_host, kept_len_host, q_obs_dev, k_layers_dev, v_layers_dev,
+                            k_out_dev, v_out_dev, window_idx_dev, kept_len_dev, keep_capacity, workspace,
+                            stream=None) -> None:
+    """Host-buffer entry: copies in, compresses, copies out, synchronises (host tensors: torch CPU, pinned)."""
+    nbytes = lambda t: t.numel() * t.element_size()
+    _check(lib().wkv_compress_group_host(
+        ctypes.byref(prob.shape), len(k_layers_host), _ptr(q_obs_host), nbytes(q_obs_host),
+        _ptr_array(k_layers_host), _ptr_array(v_layers_host), nbytes(k_layers_host[0]),
+        _ptr_array(k_out_host), _ptr_array(v_out_host), nbytes(k_out_host[0]),
+        _ptr(window_idx_host), _ptr(kept_len_host), _ptr(q_obs_dev), _ptr_array(k_layers_dev),
+        _ptr_array(v_layers_dev), _ptr_array(k_out_dev), _ptr_array(v_out_dev), _ptr(window_idx_dev),
+        _ptr(kept_len_dev), keep_capacity, _ptr(workspace), workspace.numel(), _stream(stream)),
+        "wkv_compress_group_host")
+
+
+def wkv_launch_count() -> int:
+    return int(lib().wkv_launch_count())
+
+
+def to_device(x: np.ndarray, device=None):
+    """numpy workload tensor (float32, or bf16 bits as uint16) -> torch CUDA tensor of that dtype."""
+    import torch
+    if x.dtype == np.uint16:
+        t = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16)
+    else:
+        t = torch.from_numpy(x)
+    return t.to(device if device is not None else "cuda")
+
+
+def to_host_bits(t) -> np.ndarray:
+    """torch tensor -> numpy array in the workload convention (bf16 as uint16 bits)."""
+    import torch
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()

@@ -1,0 +1,470 @@
+// Host side of the C ABI: argument validation, shape resolution, workspace
+// carve-up and kernel sequencing.  No device memory is allocated here.
+#include "wkv_internal.cuh"
+
+#include <atomic>
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+namespace wkv {
+
+static thread_local char g_detail[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+void set_error_detail(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_detail, sizeof g_detail, fmt, ap);
+    va_end(ap);
+}
+
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+size_t score_simt_smem_bytes(const KShape &ks, int r_pad);
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+Workspace plan_workspace(const KShape &ks)
+{
+    Workspace w;
+    const size_t units = (size_t)ks.batch * ks.hkv;
+    w.r_pad = (ks.R + 63) / 64 * 64;
+    w.n_stat_chunks = (ks.max_seqlen + kStatChunk - 1) / kStatChunk;
+    size_t off = 0;
+    w.stats_off = off;
+    off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
+    w.lse_off = off;
+    off = align_up(off + units * w.r_pad * sizeof(float), 256);
+    w.scores_off = off;
+    off = align_up(off + units * (size_t)ks.kw_max * sizeof(float), 256);
+    w.total = off;
+    return w;
+}
+
+static int elem_bytes(int dtype) { return dtype == WKV_F32 ? 4 : 2; }
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the shape and fills the kernel-side copy.  `seqlens` are read from the host arrays.
+static int resolve(const wkv_shape *s, KShape &ks)
+{
+    if (!s) {
+        set_error_detail("shape is NULL");
+        return WKV_ERR_NULL;
+    }
+    if (s->struct_size != sizeof(wkv_shape)) {
+        set_error_detail("struct_size %u != %zu", s->struct_size, sizeof(wkv_shape));
+        return WKV_ERR_SHAPE;
+    }
+    if (s->dtype != WKV_F32 && s->dtype != WKV_BF16) {
+        set_error_detail("dtype %d unknown", s->dtype);
+        return WKV_ERR_DTYPE;
+    }
+    if (s->batch < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->head_dim < 1 || s->l_obs < 1 ||
+        s->window < 1 || s->max_seqlen < 1 || s->top_p < 0) {
+        set_error_detail("non-positive size (batch %d, heads %d/%d, d %d, alpha %d, omega %d, N %d, p %d)",
+                         s->batch, s->n_q_heads, s->n_kv_heads, s->head_dim, s->l_obs, s->window,
+                         s->max_seqlen, s->top_p);
+        return WKV_ERR_SHAPE;
+    }
+    if (s->n_q_heads % s->n_kv_heads) {
+        set_error_detail("n_q_heads %d not a multiple of n_kv_heads %d", s->n_q_heads, s->n_kv_heads);
+        return WKV_ERR_SHAPE;
+    }
+    if (s->task != WKV_TASK_LOCALIZATION && s->task != WKV_TASK_AGGREGATION) {
+        set_error_detail("task %d unknown", s->task);
+        return WKV_ERR_SHAPE;
+    }
+    if (s->score_impl < WKV_SCORE_AUTO || s->score_impl > WKV_SCORE_TCGEN05 || s->reserved != 0) {
+        set_error_detail("score_impl %d / reserved %d invalid", s->score_impl, s->reserved);
+        return WKV_ERR_SHAPE;
+    }
+    const int eb = elem_bytes(s->dtype);
+    if ((s->head_dim * eb) % 16) {
+        set_error_detail("head_dim %d: a row must be a multiple of 16 bytes", s->head_dim);
+        return WKV_ERR_ALIGN;
+    }
+    const int64_t strides[6] = {s->stride_b, s->stride_h, s->stride_t,
+                                s->q_stride_b, s->q_stride_h, s->q_stride_t};
+    for (int i = 0; i < 6; ++i) {
+        if (strides[i] < 0 || (strides[i] * eb) % 16) {
+            set_error_detail("stride #%d = %lld is negative or not 16-byte aligned", i, (long long)strides[i]);
+            return WKV_ERR_ALIGN;
+        }
+    }
+    if (s->stride_t < s->head_dim || s->q_stride_t < s->head_dim) {
+        set_error_detail("token stride smaller than head_dim");
+        return WKV_ERR_SHAPE;
+    }
+    if ((s->cu_seqlens_host == nullptr) != (s->cu_seqlens_dev == nullptr) ||
+        (s->budgets_host == nullptr) != (s->budgets_dev == nullptr)) {
+        set_error_detail("host and device copies of cu_seqlens / budgets must be given together");
+        return WKV_ERR_NULL;
+    }
+    long long total = 0;
+    int kw_max = 1, k_max = 1, nr_max = 1;
+    for (int b = 0; b < s->batch; ++b) {
+        int n = s->max_seqlen;
+        if (s->cu_seqlens_host) {
+            n = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
+            if (n < 1 || n > s->max_seqlen || (b == 0 && s->cu_seqlens_host[0] != 0)) {
+                set_error_detail("cu_seqlens: sequence %d has length %d (max_seqlen %d)", b, n, s->max_seqlen);
+                return WKV_ERR_SHAPE;
+            }
+        }
+        total += n;
+        const int budget = s->budgets_host ? s->budgets_host[b] : s->budget;
+        if (budget < 0) {
+            set_error_detail("budget of sequence %d is negative (%d)", b, budget);
+            return WKV_ERR_BUDGET;
+        }
+        const int kw = num_windows(n, s->l_obs, s->window);
+        const int k = num_selected(n, s->l_obs, s->window, budget);
+        if (kw > kw_max) kw_max = kw;
+        if (k > k_max) k_max = k;
+        if (n - s->l_obs > nr_max) nr_max = n - s->l_obs;
+    }
+    if (total > 0x7fffffffLL) {
+        set_error_detail("more than 2^31-1 tokens in the batch");
+        return WKV_ERR_LIMIT;
+    }
+    ks.batch = s->batch;
+    ks.hq = s->n_q_heads;
+    ks.hkv = s->n_kv_heads;
+    ks.d = s->head_dim;
+    ks.alpha = s->l_obs;
+    ks.omega = s->window;
+    ks.p = s->task == WKV_TASK_LOCALIZATION ? s->window : (s->top_p > 0 ? s->top_p : (s->window + 1) / 2);
+    ks.max_seqlen = s->max_seqlen;
+    ks.budget = s->budget;
+    ks.G = s->n_q_heads / s->n_kv_heads;
+    ks.R = ks.G * ks.alpha;
+    ks.kw_max = kw_max;
+    ks.k_max = k_max;
+    ks.nr_max = s->max_seqlen - s->l_obs > 1 ? s->max_seqlen - s->l_obs : 1;
+    (void)nr_max;
+    ks.cu = s->cu_seqlens_dev;
+    ks.budgets = s->budgets_dev;
+    ks.sb = s->stride_b;
+    ks.sh = s->stride_h;
+    ks.st = s->stride_t;
+    ks.qsb = s->q_stride_b;
+    ks.qsh = s->q_stride_h;
+    ks.qst = s->q_stride_t;
+    ks.scale_log2 = (float)(1.4426950408889634 / sqrt((double)s->head_dim));
+    return WKV_OK;
+}
+
+static int check_cuda(cudaError_t e, const char *what)
+{
+    if (e == cudaSuccess) return WKV_OK;
+    set_error_detail("%s: %s", what, cudaGetErrorString(e));
+    return WKV_ERR_CUDA;
+}
+
+static int check_workspace(const Workspace &ws, const void *workspace, size_t bytes)
+{
+    if (!workspace) {
+        set_error_detail("workspace is NULL (%zu bytes needed)", ws.total);
+        return WKV_ERR_WORKSPACE;
+    }
+    if (bytes < ws.total) {
+        set_error_detail("workspace has %zu bytes, %zu needed", bytes, ws.total);
+        return WKV_ERR_WORKSPACE;
+    }
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) {
+        set_error_detail("workspace is not 256-byte aligned");
+        return WKV_ERR_WORKSPACE;
+    }
+    return WKV_OK;
+}
+
+// picks the kernel family; returns a status
+static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace &ws, bool &use_tc)
+{
+    const bool tc_ok = score_tc_supported(ks, s->dtype);
+    if (s->score_impl == WKV_SCORE_TCGEN05 && !tc_ok) {
+        set_error_detail("tensor-core score kernels need bf16, head_dim 64/128 and G*alpha <= 256");
+        return WKV_ERR_UNSUPPORTED;
+    }
+    use_tc = tc_ok && s->score_impl != WKV_SCORE_SIMT;
+    if (!use_tc) {
+        const size_t need = score_simt_smem_bytes(ks, ws.r_pad);
+        if (need > 227u * 1024u) {
+            set_error_detail("CUDA-core score kernels need %zu bytes of shared memory (> 227 KB): "
+                             "G*alpha*head_dim too large", need);
+            return WKV_ERR_UNSUPPORTED;
+        }
+    }
+    return WKV_OK;
+}
+
+static int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
+                    float *window_scores, float *token_scores, void *workspace, cudaStream_t stream)
+{
+    if (!aligned16(q) || !aligned16(k)) {
+        set_error_detail("q_obs / k_leader not 16-byte aligned");
+        return WKV_ERR_ALIGN;
+    }
+    bool use_tc = false;
+    int st = pick_score_impl(s, ks, ws, use_tc);
+    if (st != WKV_OK) return st;
+    if (use_tc) return launch_score_tc(ks, q, k, window_scores, token_scores, workspace, ws, stream);
+    return check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream),
+                      "score kernels");
+}
+
+static int fill_table(int n_layers, const void *const *k_layers, const void *const *v_layers,
+                      void *const *k_out, void *const *v_out, LayerTable &tab, int &n_tensors)
+{
+    if (n_layers < 1 || n_layers > WKV_MAX_GROUP_LAYERS) {
+        set_error_detail("n_layers %d outside 1..%d", n_layers, WKV_MAX_GROUP_LAYERS);
+        return WKV_ERR_LIMIT;
+    }
+    if (!k_layers || !k_out) {
+        set_error_detail("k_layers / k_out_layers is NULL");
+        return WKV_ERR_NULL;
+    }
+    const bool with_v = v_layers && v_out;
+    n_tensors = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const void *src[2] = {k_layers[l], with_v ? v_layers[l] : nullptr};
+        void *dst[2] = {k_out[l], with_v ? v_out[l] : nullptr};
+        for (int t = 0; t < (with_v ? 2 : 1); ++t) {
+            if (!src[t] || !dst[t]) {
+                set_error_detail("layer %d: NULL tensor pointer", l);
+                return WKV_ERR_NULL;
+            }
+            if (!aligned16(src[t]) || !aligned16(dst[t])) {
+                set_error_detail("layer %d: tensor pointer not 16-byte aligned", l);
+                return WKV_ERR_ALIGN;
+            }
+            tab.src[n_tensors] = src[t];
+            tab.dst[n_tensors] = dst[t];
+            ++n_tensors;
+        }
+    }
+    return WKV_OK;
+}
+
+static int keep_max_of(const wkv_shape *s)
+{
+    int best = 0;
+    for (int b = 0; b < s->batch; ++b) {
+        const int n = s->cu_seqlens_host ? s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b] : s->max_seqlen;
+        const int budget = s->budgets_host ? s->budgets_host[b] : s->budget;
+        const int rows = num_selected(n, s->l_obs, s->window, budget) * s->window + (n < s->l_obs ? n : s->l_obs);
+        if (rows > best) best = rows;
+    }
+    return best;
+}
+
+}  // namespace wkv
+
+using namespace wkv;
+
+extern "C" {
+
+int32_t wkv_num_windows(int32_t n, int32_t alpha, int32_t omega) { return num_windows(n, alpha, omega); }
+
+int32_t wkv_num_selected(int32_t n, int32_t alpha, int32_t omega, int32_t budget)
+{
+    return num_selected(n, alpha, omega, budget);
+}
+
+int32_t wkv_kw_max(const wkv_shape *s)
+{
+    KShape ks;
+    return resolve(s, ks) == WKV_OK ? ks.kw_max : 0;
+}
+
+int32_t wkv_k_max(const wkv_shape *s)
+{
+    KShape ks;
+    return resolve(s, ks) == WKV_OK ? ks.k_max : 0;
+}
+
+int32_t wkv_keep_max(const wkv_shape *s)
+{
+    KShape ks;
+    return resolve(s, ks) == WKV_OK ? keep_max_of(s) : 0;
+}
+
+size_t wkv_workspace_bytes(const wkv_shape *s)
+{
+    KShape ks;
+    if (resolve(s, ks) != WKV_OK) return 0;
+    return plan_workspace(ks).total;
+}
+
+int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader, float *window_scores,
+                      float *token_scores, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!q_obs || !k_leader || !window_scores) {
+        set_error_detail("q_obs / k_leader / window_scores is NULL");
+        return WKV_ERR_NULL;
+    }
+    const Workspace ws = plan_workspace(ks);
+    st = check_workspace(ws, workspace, workspace_bytes);
+    if (st != WKV_OK) return st;
+    return do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, workspace,
+                    static_cast<cudaStream_t>(cuda_stream));
+}
+
+int wkv_select_topk_windows(const wkv_shape *s, const float *window_scores, int32_t *window_idx,
+                            int32_t *kept_len, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!window_scores || !window_idx || !kept_len) {
+        set_error_detail("window_scores / window_idx / kept_len is NULL");
+        return WKV_ERR_NULL;
+    }
+    return check_cuda(launch_topk(ks, window_scores, window_idx, kept_len, static_cast<cudaStream_t>(cuda_stream)),
+                      "selection kernel");
+}
+
+int wkv_gather_kv(const wkv_shape *s, int32_t n_layers, const void *const *k_layers,
+                  const void *const *v_layers, const int32_t *window_idx, void *const *k_out_layers,
+                  void *const *v_out_layers, const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                  void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!window_idx) {
+        set_error_detail("window_idx is NULL");
+        return WKV_ERR_NULL;
+    }
+    LayerTable tab;
+    int n_tensors = 0;
+    st = fill_table(n_layers, k_layers, v_layers, k_out_layers, v_out_layers, tab, n_tensors);
+    if (st != WKV_OK) return st;
+    if (!cu_seqlens_out && keep_capacity < keep_max_of(s)) {
+        set_error_detail("keep_capacity %d smaller than the %d rows a unit may keep", keep_capacity, keep_max_of(s));
+        return WKV_ERR_SHAPE;
+    }
+    return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
+                                    keep_capacity, static_cast<cudaStream_t>(cuda_stream)),
+                      "gather kernel");
+}
+
+int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
+                       const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
+                       void *const *v_out_layers, float *window_scores, int32_t *window_idx,
+                       int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!q_obs_leader || !window_idx || !kept_len) {
+        set_error_detail("q_obs_leader / window_idx / kept_len is NULL");
+        return WKV_ERR_NULL;
+    }
+    LayerTable tab;
+    int n_tensors = 0;
+    st = fill_table(n_layers, k_layers, v_layers, k_out_layers, v_out_layers, tab, n_tensors);
+    if (st != WKV_OK) return st;
+    if (!cu_seqlens_out && keep_capacity < keep_max_of(s)) {
+        set_error_detail("keep_capacity %d smaller than the %d rows a unit may keep", keep_capacity, keep_max_of(s));
+        return WKV_ERR_SHAPE;
+    }
+    const Workspace ws = plan_workspace(ks);
+    st = check_workspace(ws, workspace, workspace_bytes);
+    if (st != WKV_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    float *scores = window_scores ? window_scores
+                                  : reinterpret_cast<float *>(static_cast<char *>(workspace) + ws.scores_off);
+    st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, workspace, stream);
+    if (st != WKV_OK) return st;
+    st = check_cuda(launch_topk(ks, scores, window_idx, kept_len, stream), "selection kernel");
+    if (st != WKV_OK) return st;
+    return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
+                                    keep_capacity, stream),
+                      "gather kernel");
+}
+
+int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers, const void *q_obs_host, size_t q_bytes,
+                            const void *const *k_layers_host, const void *const *v_layers_host,
+                            size_t bytes_per_layer, void *const *k_out_layers_host,
+                            void *const *v_out_layers_host, size_t out_bytes_per_layer,
+                            int32_t *window_idx_host, int32_t *kept_len_host, void *q_obs_dev,
+                            void *const *k_layers_dev, void *const *v_layers_dev,
+                            void *const *k_out_layers_dev, void *const *v_out_layers_dev,
+                            int32_t *window_idx_dev, int32_t *kept_len_dev, int32_t keep_capacity,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (n_layers < 1 || n_layers > WKV_MAX_GROUP_LAYERS) {
+        set_error_detail("n_layers %d outside 1..%d", n_layers, WKV_MAX_GROUP_LAYERS);
+        return WKV_ERR_LIMIT;
+    }
+    if (!q_obs_host || !k_layers_host || !v_layers_host || !k_out_layers_host || !v_out_layers_host ||
+        !window_idx_host || !kept_len_host || !q_obs_dev || !k_layers_dev || !v_layers_dev ||
+        !k_out_layers_dev || !v_out_layers_dev || !window_idx_dev || !kept_len_dev) {
+        set_error_detail("a host or staging pointer is NULL");
+        return WKV_ERR_NULL;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = check_cuda(cudaMemcpyAsync(q_obs_dev, q_obs_host, q_bytes, cudaMemcpyHostToDevice, stream), "copy of q_obs");
+    for (int l = 0; l < n_layers && st == WKV_OK; ++l) {
+        st = check_cuda(cudaMemcpyAsync(k_layers_dev[l], k_layers_host[l], bytes_per_layer,
+                                        cudaMemcpyHostToDevice, stream), "copy of K");
+        if (st == WKV_OK)
+            st = check_cuda(cudaMemcpyAsync(v_layers_dev[l], v_layers_host[l], bytes_per_layer,
+                                            cudaMemcpyHostToDevice, stream), "copy of V");
+    }
+    if (st != WKV_OK) return st;
+    st = wkv_compress_group(s, n_layers, q_obs_dev, k_layers_dev, v_layers_dev, k_out_layers_dev,
+                            v_out_layers_dev, nullptr, window_idx_dev, kept_len_dev, nullptr, keep_capacity,
+                            workspace, workspace_bytes, cuda_stream);
+    if (st != WKV_OK) return st;
+    const size_t units = (size_t)ks.batch * ks.hkv;
+    st = check_cuda(cudaMemcpyAsync(window_idx_host, window_idx_dev, units * ks.k_max * sizeof(int32_t),
+                                    cudaMemcpyDeviceToHost, stream), "copy of window_idx");
+    if (st == WKV_OK)
+        st = check_cuda(cudaMemcpyAsync(kept_len_host, kept_len_dev, units * sizeof(int32_t),
+                                        cudaMemcpyDeviceToHost, stream), "copy of kept_len");
+    for (int l = 0; l < n_layers && st == WKV_OK; ++l) {
+        st = check_cuda(cudaMemcpyAsync(k_out_layers_host[l], k_out_layers_dev[l], out_bytes_per_layer,
+                                        cudaMemcpyDeviceToHost, stream), "copy of compact K");
+        if (st == WKV_OK)
+            st = check_cuda(cudaMemcpyAsync(v_out_layers_host[l], v_out_layers_dev[l], out_bytes_per_layer,
+                                            cudaMemcpyDeviceToHost, stream), "copy of compact V");
+    }
+    if (st != WKV_OK) return st;
+    return check_cuda(cudaStreamSynchronize(stream), "stream synchronisation");
+}
+
+const char *wkv_status_string(int status)
+{
+    switch (status) {
+    case WKV_OK: return "ok";
+    case WKV_ERR_NULL: return "required pointer is NULL";
+    case WKV_ERR_SHAPE: return "invalid shape";
+    case WKV_ERR_DTYPE: return "invalid dtype";
+    case WKV_ERR_BUDGET: return "invalid budget";
+    case WKV_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+    case WKV_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case WKV_ERR_UNSUPPORTED: return "shape not supported by the kernels";
+    case WKV_ERR_CUDA: return "CUDA call failed";
+    case WKV_ERR_LIMIT: return "size beyond a fixed maximum";
+    default: return "unknown status";
+    }
+}
+
+const char *wkv_last_error_detail(void) { return g_detail; }
+
+uint64_t wkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

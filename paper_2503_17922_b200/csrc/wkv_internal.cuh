@@ -1,0 +1,98 @@
+// Internal declarations shared by the library's translation units (host side of
+// the C ABI and the kernel launchers).  Not part of the public interface.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "wkv.h"
+
+namespace wkv {
+
+// Shape as the kernels see it: plain values, device pointers only.
+struct KShape {
+    int batch, hq, hkv, d;
+    int alpha, omega, p;       // p already resolved from task/top_p (Eq. 4)
+    int max_seqlen, budget;
+    int G, R;                  // query heads per KV head; observation rows per unit = G*alpha
+    int kw_max, k_max, nr_max; // leading sizes of window_scores / window_idx / token_scores
+    const int *cu;             // device cu_seqlens or nullptr
+    const int *budgets;        // device budgets or nullptr
+    long long sb, sh, st;      // K/V element strides
+    long long qsb, qsh, qst;   // Q_obs element strides
+    float scale_log2;          // log2(e)/sqrt(d): logits are handled in base 2
+};
+
+// Per-sequence integers, the same formulas on host and device (Eq. 3 and the
+// budget sentence after Eq. 4).
+__host__ __device__ inline int num_windows(int n, int alpha, int omega)
+{
+    return n <= alpha ? 0 : (n - alpha + omega - 1) / omega;
+}
+__host__ __device__ inline int num_selected(int n, int alpha, int omega, int budget)
+{
+    int kw = num_windows(n, alpha, omega);
+    int k = budget > alpha ? (budget - alpha) / omega : 0;
+    return k < kw ? k : kw;
+}
+
+struct SeqInfo {
+    int n;          // context length
+    long long off;  // first row of the sequence in the packed layout (0 when dense)
+    int budget;
+};
+
+__device__ inline SeqInfo seq_info(const KShape &s, int b)
+{
+    SeqInfo r;
+    if (s.cu) {
+        int lo = s.cu[b];
+        r.n = s.cu[b + 1] - lo;
+        r.off = lo;
+    } else {
+        r.n = s.max_seqlen;
+        r.off = 0;
+    }
+    r.budget = s.budgets ? s.budgets[b] : s.budget;
+    return r;
+}
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct Workspace {
+    size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
+    size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
+    size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none
+    size_t total;
+    int n_stat_chunks;
+    int r_pad;
+};
+
+constexpr int kStatChunk = 512;   // keys per partial-statistics chunk (both kernel families)
+
+Workspace plan_workspace(const KShape &ks);
+
+// Launchers (each returns a cudaError_t from the launch).
+cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const void *k,
+                              float *window_scores, float *token_scores,
+                              void *workspace, const Workspace &ws, cudaStream_t stream);
+bool score_tc_supported(const KShape &ks, int dtype);
+int launch_score_tc(const KShape &ks, const void *q, const void *k,
+                    float *window_scores, float *token_scores,
+                    void *workspace, const Workspace &ws, cudaStream_t stream);
+cudaError_t launch_topk(const KShape &ks, const float *window_scores, int *window_idx, int *kept_len,
+                        cudaStream_t stream);
+
+struct LayerTable {
+    const void *src[2 * WKV_MAX_GROUP_LAYERS];
+    void *dst[2 * WKV_MAX_GROUP_LAYERS];
+};
+cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const LayerTable &tab,
+                          const int *window_idx, const int *cu_out, int keep_capacity,
+                          cudaStream_t stream);
+
+void count_launches(int n);
+void set_error_detail(const char *fmt, ...);
+
+}  // namespace wkv

@@ -1,0 +1,275 @@
+"""GPU parity tests: the CUDA library (through the C ABI) against the CPU oracle on
+the same seeded inputs.  Index and gathered-KV checks are exact (up to the stated
+near-tie rule), pooled scores within 1e-3 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_17922_b200 import binding
+from paper_2503_17922_b200 import workloads as wl
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = {"simt": binding.WKV_SCORE_SIMT, "auto": binding.WKV_SCORE_AUTO}
+
+
+def small(dtype="bf16", **kw):
+    """A small case that still spans several key tiles, several chunks and a ragged tail."""
+    base = dict(name="small", dtype=dtype, batch=2, n_layers=2, gamma=2, n_q_heads=8, n_kv_heads=2,
+                head_dim=128, max_seqlen=1337, l_obs=16, window=8, top_p=4, budget_frac=0.2,
+                n_planted=5, config_id=9)
+    base.update(kw)
+    return wl.scaled(wl.llama8b_single_group(), **base)
+
+
+# ------------------------------------------------------------------ whole path, small shapes
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("case", [
+    dict(),                                                   # bf16, R = 64, ragged last window
+    dict(task=wl.TASK_AGGREGATION, top_p=3),
+    dict(task=wl.TASK_AGGREGATION, top_p=1, window=16),
+    dict(task=wl.TASK_AGGREGATION, top_p=31, window=32, l_obs=32),   # R = 128
+    dict(head_dim=64, window=4, l_obs=8),                     # R = 32
+    dict(n_q_heads=8, n_kv_heads=1, l_obs=32, max_seqlen=2100),       # R = 256
+    dict(n_q_heads=6, n_kv_heads=2, l_obs=5, window=7, max_seqlen=999),   # odd sizes: R = 15, omega = 7
+    dict(max_seqlen=4096 + 16, window=16, budget_frac=0.12),  # review length a multiple of everything
+    dict(dtype="f32", head_dim=64, n_q_heads=4, l_obs=8),     # fp32 inputs
+    dict(ragged=True, batch=4, max_seqlen=1500),              # packed layout, n_b in [750, 1500]
+    dict(ragged=True, batch=3, max_seqlen=700, task=wl.TASK_AGGREGATION, top_p=2, dtype="f32", head_dim=64),
+], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()) or "base")
+def test_group_small(case, impl):
+    w = small(**case)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=IMPLS[impl])
+    assert max_rel < 1e-4           # far inside the 1e-3 bar; a loose bound here would hide a bug
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            planted = wl.planted_windows(w, b, h, int(grp["seqlens"][b]))
+            k = oracle.num_selected(int(grp["seqlens"][b]), w.l_obs, w.window, int(grp["budgets"][b]))
+            if len(planted) <= k:
+                assert set(planted) <= set(gpu["window_idx"][b, h, :k].tolist())
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+def test_stage_entry_points_and_token_scores(impl):
+    w = small(max_seqlen=1100)
+    grp = wl.make_group(w, 0)
+    ref = oracle.select_leader(grp["q_obs"], grp["k_layers"][0], want_tokens=True, **pu.oracle_kwargs(w, grp))
+    gpu = pu.run_gpu_group(w, grp, score_impl=IMPLS[impl], staged=True, want_tokens=True)
+    pu.check_selection(w, grp, gpu, ref)
+    pu.check_gather(w, grp, gpu)
+    n_r = w.max_seqlen - w.l_obs
+    t_ref = ref["token_scores"][:, :, :n_r]
+    t_gpu = gpu["token_scores"][:, :, :n_r].astype(np.float64)
+    rel = np.abs(t_gpu - t_ref) / t_ref
+    assert rel.max() < 1e-4
+
+
+def test_same_result_twice_and_across_entry_points():
+    w = small()
+    grp = wl.make_group(w, 0)
+    a = pu.run_gpu_group(w, grp)
+    b = pu.run_gpu_group(w, grp)
+    c = pu.run_gpu_group(w, grp, staged=True)
+    for x in (b, c):
+        np.testing.assert_array_equal(a["window_scores"][..., : a["prob"].kw_max], x["window_scores"][..., : a["prob"].kw_max])
+        np.testing.assert_array_equal(a["window_idx"], x["window_idx"])
+        np.testing.assert_array_equal(a["k_out"][1], x["k_out"][1])
+
+
+# ------------------------------------------------------------------ selection, exact
+@pytest.mark.parametrize("kw_n,budget", [(40, 100), (127, 128), (1020, 983), (5000, 2048), (9000, 40000), (1, 64)])
+def test_selection_bit_exact_on_given_scores(kw_n, budget):
+    # feed the same fp32 scores to both sides: indices must agree exactly, including ties
+    alpha, omega = 8, 8
+    n = alpha + kw_n * omega - 3            # ragged last window
+    B, H = 2, 3
+    g = np.random.Generator(np.random.Philox(key=77 + kw_n))
+    scores = g.standard_normal((B, H, kw_n)).astype(np.float32)
+    scores[0, 1] = np.round(scores[0, 1] * 2) / 2            # many exact ties
+    scores[1, 0] = 0.25                                       # all equal
+    scores[1, 1, ::3] = -0.0
+    scores[1, 1, 1::3] = 0.0                                  # signed zeros compare equal
+    scores[1, 2] = np.abs(scores[1, 2]) * 1e-30               # tiny positive values
+    prob = binding.Problem(dtype="bf16", batch=B, n_q_heads=H, n_kv_heads=H, head_dim=64, l_obs=alpha,
+                           window=omega, task=0, top_p=0, max_seqlen=n, budgets=[budget] * B)
+    assert prob.kw_max == kw_n
+    d_scores = torch.from_numpy(scores).cuda()
+    idx = torch.full((B, H, prob.k_max), -9, dtype=torch.int32, device="cuda")
+    kept = torch.full((B, H), -9, dtype=torch.int32, device="cuda")
+    binding.wkv_select_topk_windows(prob, d_scores, idx, kept)
+    torch.cuda.synchronize()
+    k = oracle.num_selected(n, alpha, omega, budget)
+    for b in range(B):
+        for h in range(H):
+            exp = oracle.select_topk(scores[b, h], k)
+            got = idx[b, h].cpu().numpy()
+            np.testing.assert_array_equal(got[:k], exp)
+            assert (got[k:] == -1).all()
+            rows = k * omega - (3 if (k and exp[-1] == kw_n - 1) else 0) + alpha
+            assert int(kept[b, h]) == rows
+
+
+# ------------------------------------------------------------------ gather, exact
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64), ("bf16", 8)])
+@pytest.mark.parametrize("packed_out", [False, True])
+def test_gather_with_given_indices(dtype, d, packed_out):
+    w = small(dtype=dtype, head_dim=d, ragged=True, batch=3, max_seqlen=900, n_layers=3, gamma=3)
+    grp = wl.make_group(w, 0)
+    prob = binding.Problem.from_workload(w)
+    # indices chosen by the test (not by either implementation): every 3rd window + the last one
+    idx = np.full((w.batch, w.n_kv_heads, prob.k_max), -1, dtype=np.int32)
+    for b in range(w.batch):
+        n = int(grp["seqlens"][b])
+        kw = oracle.num_windows(n, w.l_obs, w.window)
+        k = oracle.num_selected(n, w.l_obs, w.window, int(grp["budgets"][b]))
+        for h in range(w.n_kv_heads):
+            cand = np.unique(np.concatenate([np.arange(h, kw, 3)[: k - 1], [kw - 1]]))[:k]
+            idx[b, h, : len(cand)] = cand
+            assert len(cand) == k
+    cap = prob.keep_max
+    cu_out = None
+    if packed_out:
+        cu_out = np.zeros(w.batch + 1, dtype=np.int32)
+        cu_out[1:] = np.cumsum([oracle.num_selected(int(n), w.l_obs, w.window, int(bb)) * w.window + w.l_obs
+                                for n, bb in zip(grp["seqlens"], grp["budgets"])])
+    ks = [binding.to_device(x) for x in grp["k_layers"]]
+    vs = [binding.to_device(x) for x in grp["v_layers"]]
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    shape = (int(cu_out[-1]), w.n_kv_heads, d) if packed_out else (w.batch, w.n_kv_heads, cap, d)
+    outs = [[torch.empty(shape, dtype=tdt, device="cuda") for _ in range(w.gamma)] for _ in range(2)]
+    for t in outs[0] + outs[1]:
+        t.view(torch.uint8).fill_(pu.FILL_BYTE)
+    binding.wkv_gather_kv(prob, ks, vs, torch.from_numpy(idx).cuda(), outs[0], outs[1],
+                          cu_seqlens_out=None if cu_out is None else torch.from_numpy(cu_out).cuda(),
+                          keep_capacity=cap)
+    torch.cuda.synchronize()
+    kw_ = dict(n_kv_heads=w.n_kv_heads, l_obs=w.l_obs, window=w.window, max_seqlen=w.max_seqlen,
+               budgets=grp["budgets"], keep_max=cap, cu_seqlens=grp["cu_seqlens"], cu_seqlens_out=cu_out,
+               fill=pu.fill_pattern(dtype))
+    for layer in range(w.gamma):
+        np.testing.assert_array_equal(binding.to_host_bits(outs[0][layer]), oracle.gather_layer(grp["k_layers"][layer], idx, **kw_))
+        np.testing.assert_array_equal(binding.to_host_bits(outs[1][layer]), oracle.gather_layer(grp["v_layers"][layer], idx, **kw_))
+
+
+# ------------------------------------------------------------------ degenerate cases
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("case", [
+    dict(budget_frac=None, budget_tokens=10 ** 6),            # budget above n: identity copy
+    dict(budget_frac=None, budget_tokens=3),                  # budget below alpha: observation rows only
+    dict(budget_frac=None, budget_tokens=16),                 # budget == alpha: k = 0
+    dict(max_seqlen=17, budget_frac=None, budget_tokens=24),  # a single review token
+    dict(max_seqlen=16, budget_frac=None, budget_tokens=24),  # n == alpha: no review context
+    dict(max_seqlen=9, budget_frac=None, budget_tokens=24),   # n < alpha
+    dict(max_seqlen=16 + 8, budget_frac=None, budget_tokens=24),  # exactly one full window
+], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
+def test_degenerate_sizes(case, impl):
+    w = small(n_planted=0, **case)
+    grp, ref, gpu, _ = pu.full_check(w, score_impl=IMPLS[impl])
+    if case.get("budget_tokens") == 10 ** 6:
+        n = w.max_seqlen
+        assert (gpu["kept_len"] == n).all()
+        np.testing.assert_array_equal(gpu["k_out"][0][:, :, :n], grp["k_layers"][0])
+
+
+def test_ragged_batch_with_a_tiny_sequence():
+    # one sequence shorter than the observation window inside a packed batch
+    w = small(ragged=True, batch=3, max_seqlen=600, n_planted=0)
+    grp = wl.make_group(w, 0)
+    cu = np.array([0, 600, 610, 610 + 433], dtype=np.int32)
+    total = int(cu[-1])
+    grp["cu_seqlens"] = cu
+    grp["seqlens"] = np.diff(cu)
+    grp["budgets"] = np.array([90, 90, 60], dtype=np.int32)
+    grp["k_layers"] = [x[:total].copy() for x in grp["k_layers"]]
+    grp["v_layers"] = [x[:total].copy() for x in grp["v_layers"]]
+    prob = binding.Problem(dtype=w.dtype, batch=3, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                           head_dim=w.head_dim, l_obs=w.l_obs, window=w.window, task=w.task, top_p=w.top_p,
+                           max_seqlen=600, budgets=grp["budgets"], cu_seqlens=cu)
+    ref = oracle.compress_group(grp["q_obs"], grp["k_layers"], grp["v_layers"], fill=pu.fill_pattern(w.dtype),
+                                **pu.oracle_kwargs(w, grp))
+    q = binding.to_device(grp["q_obs"])
+    ks = [binding.to_device(x) for x in grp["k_layers"]]
+    vs = [binding.to_device(x) for x in grp["v_layers"]]
+    out = prob.alloc_outputs(len(ks), fill_byte=pu.FILL_BYTE)
+    binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
+                               out["window_idx"], out["kept_len"], prob.alloc_workspace(),
+                               keep_capacity=out["keep_capacity"])
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out["kept_len"].cpu().numpy(), ref["kept_len"])
+    assert ref["kept_len"][1, 0] == 10
+    np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), ref["window_idx"])
+    for layer in range(len(ks)):
+        np.testing.assert_array_equal(binding.to_host_bits(out["k_out"][layer]), ref["k_out"][layer])
+        np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][layer]), ref["v_out"][layer])
+
+
+def test_launches_are_counted_and_errors_raise():
+    w = small()
+    before = binding.wkv_launch_count()
+    pu.run_gpu_group(w, wl.make_group(w, 0))
+    assert binding.wkv_launch_count() - before >= 3
+    prob = binding.Problem.from_workload(w)
+    with pytest.raises(binding.WkvError):
+        binding.wkv_score_windows(prob, None, None, None, None, prob.alloc_workspace())
+
+
+# ------------------------------------------------------------------ the five configurations, full size
+def test_config1_tiny_fp32():
+    w = wl.tiny()
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w)
+    assert gpu["prob"].k_max == 15 and gpu["prob"].keep_max == 128
+    for h in range(w.n_kv_heads):
+        assert set(wl.planted_windows(w, 0, h, 1024)) <= set(gpu["window_idx"][0, h].tolist())
+
+
+@pytest.mark.parametrize("task", [wl.TASK_LOCALIZATION, wl.TASK_AGGREGATION])
+def test_config2_llama8b_single_group(task):
+    w = wl.llama8b_single_group(task)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w)
+    assert gpu["prob"].k_max == 118 and gpu["prob"].keep_max == 976
+    for h in range(w.n_kv_heads):
+        assert set(wl.planted_windows(w, 0, h, 8192)) <= set(gpu["window_idx"][0, h].tolist())
+
+
+@pytest.mark.parametrize("group", [0, 5])
+def test_config3_llama8b_32k(group):
+    w = wl.llama8b_full()
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=group)
+    assert gpu["prob"].k_max == 243 and gpu["prob"].keep_max == 3920
+
+
+@pytest.mark.parametrize("n,depth", [(4096, 0.1), (16384, 0.5), (32768, 0.9)])
+def test_config4_needle(n, depth):
+    w = wl.mistral_needle(n, depth)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=3)
+    for h in range(w.n_kv_heads):
+        needle = wl.planted_windows(w, 0, h, n)
+        assert len(needle) == 8 and set(needle) <= set(gpu["window_idx"][0, h].tolist())
+
+
+def test_config5_batched_ragged_sampled_units():
+    # the leader's K of one group at full size (B = 8, n_b in [32K, 64K], packed); the oracle
+    # scores a sample of units, every unit's structure and gather is checked
+    w = wl.batched_ragged()
+    q_obs = wl.make_q_obs(w, 0)
+    k0, v0 = wl.make_layer_kv(w, 0, q_obs)
+    grp = {"q_obs": q_obs, "k_layers": [k0], "v_layers": [v0], "seqlens": w.seqlens(),
+           "cu_seqlens": w.cu_seqlens(), "budgets": w.budgets()}
+    units = [(0, 0), (3, 5), (7, 7), (int(np.argmin(grp["seqlens"])), 2)]
+    mask = np.zeros((w.batch, w.n_kv_heads), dtype=np.uint8)
+    for b, h in units:
+        mask[b, h] = 1
+    ref = oracle.select_leader(q_obs, k0, unit_mask=mask, **pu.oracle_kwargs(w, grp))
+    gpu = pu.run_gpu_group(w, grp)
+    pu.check_selection(w, grp, gpu, ref, units=units)
+    pu.check_gather(w, grp, gpu)
+    for b in range(w.batch):          # structure of every unit
+        n = int(grp["seqlens"][b])
+        k = oracle.num_selected(n, w.l_obs, w.window, int(grp["budgets"][b]))
+        for h in range(w.n_kv_heads):
+            sel = gpu["window_idx"][b, h, :k]
+            assert (np.diff(sel) > 0).all() and sel[0] >= 0 and sel[-1] < oracle.num_windows(n, w.l_obs, w.window)
+            assert set(wl.planted_windows(w, b, h, n)) <= set(sel.tolist())
