@@ -207,8 +207,9 @@ class Problem:
 
     # ---- caller-side allocations (torch is the allocator, nothing else) ----
     def alloc_workspace(self):
+        """Zero-filled scratch; its first int32 is the device status word (see `device_status`)."""
         import torch
-        return torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+        return torch.zeros(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
 
     def alloc_outputs(self, n_layers: int, fill_byte: Optional[int] = None, keep_capacity: Optional[int] = None):
         import torch
@@ -273,6 +274,11 @@ def wkv_compress_group_host(prob: Problem, q_obs_host, k_layers_host, v_layers_h
         _ptr_array(v_layers_dev), _ptr_array(k_out_dev), _ptr_array(v_out_dev), _ptr(window_idx_dev),
         _ptr(kept_len_dev), keep_capacity, _ptr(workspace), workspace.numel(), _stream(stream)),
         "wkv_compress_group_host")
+
+
+def device_status(workspace) -> int:
+    """The workspace's status word (synchronises): 0, or the OR of the error bits a kernel has set."""
+    return int(workspace[:4].view(__import__("torch").int32).item())
 
 
 def wkv_launch_count() -> int:

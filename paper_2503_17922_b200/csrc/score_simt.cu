@@ -176,36 +176,6 @@ score_stats_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k, flo
     }
 }
 
-// Eq. 4 for one window held in shared memory: mean of the p largest of `size` values.
-// Elements are visited in the strict order (value descending, position ascending), so
-// equal values are each taken once.
-__device__ inline float pool_top_p(const float *w, int size, int p)
-{
-    if (p >= size) {
-        float acc = 0.f;
-        for (int x = 0; x < size; ++x) acc += w[x];
-        return acc / (float)size;
-    }
-    float acc = 0.f, prev_v = INFINITY;
-    int prev_i = -1;
-    for (int round = 0; round < p; ++round) {
-        float best_v = -INFINITY;
-        int best_i = size;
-        for (int x = 0; x < size; ++x) {
-            float v = w[x];
-            bool after_prev = v < prev_v || (v == prev_v && x > prev_i);
-            if (after_prev && (v > best_v || best_i == size)) {
-                best_v = v;
-                best_i = x;
-            }
-        }
-        acc += best_v;
-        prev_v = best_v;
-        prev_i = best_i;
-    }
-    return acc / (float)p;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 score_pool_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k,

@@ -33,7 +33,11 @@ Workspace plan_workspace(const KShape &ks)
     const size_t units = (size_t)ks.batch * ks.hkv;
     w.r_pad = (ks.R + 63) / 64 * 64;
     w.n_stat_chunks = (ks.max_seqlen + kStatChunk - 1) / kStatChunk;
+    const int tc_chunks = tc_chunks_per_unit((int)units, ks.max_seqlen);
+    if (tc_chunks > w.n_stat_chunks) w.n_stat_chunks = tc_chunks;
     size_t off = 0;
+    w.status_off = off;
+    off = 256;
     w.stats_off = off;
     off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
     w.lse_off = off;
@@ -140,6 +144,7 @@ static int resolve(const wkv_shape *s, KShape &ks)
     ks.p = s->task == WKV_TASK_LOCALIZATION ? s->window : (s->top_p > 0 ? s->top_p : (s->window + 1) / 2);
     ks.max_seqlen = s->max_seqlen;
     ks.budget = s->budget;
+    ks.total_rows = (int)total;
     ks.G = s->n_q_heads / s->n_kv_heads;
     ks.R = ks.G * ks.alpha;
     ks.kw_max = kw_max;
@@ -212,7 +217,12 @@ static int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, c
     bool use_tc = false;
     int st = pick_score_impl(s, ks, ws, use_tc);
     if (st != WKV_OK) return st;
-    if (use_tc) return launch_score_tc(ks, q, k, window_scores, token_scores, workspace, ws, stream);
+    if (use_tc) {
+        st = launch_score_tc(ks, q, k, window_scores, token_scores, workspace, ws, stream);
+        // a key layout that no tensor map can describe is served by the CUDA-core kernels
+        if (st != WKV_ERR_UNSUPPORTED || s->score_impl == WKV_SCORE_TCGEN05) return st;
+        if (score_simt_smem_bytes(ks, ws.r_pad) > 227u * 1024u) return st;
+    }
     return check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream),
                       "score kernels");
 }

@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <math.h>
 #include <stdint.h>
 #include <stddef.h>
 
@@ -16,6 +17,7 @@ struct KShape {
     int batch, hq, hkv, d;
     int alpha, omega, p;       // p already resolved from task/top_p (Eq. 4)
     int max_seqlen, budget;
+    int total_rows;            // sum of the sequence lengths (rows of the packed layout)
     int G, R;                  // query heads per KV head; observation rows per unit = G*alpha
     int kw_max, k_max, nr_max; // leading sizes of window_scores / window_idx / token_scores
     const int *cu;             // device cu_seqlens or nullptr
@@ -61,6 +63,7 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
+    size_t status_off;   // int: device status word, only ever OR-ed by the kernels (0 = no error)
     size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
     size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
     size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none
@@ -69,7 +72,37 @@ struct Workspace {
     int r_pad;
 };
 
-constexpr int kStatChunk = 512;   // keys per partial-statistics chunk (both kernel families)
+constexpr int kStatChunk = 512;   // keys per partial-statistics chunk of the CUDA-core kernels
+
+// Tensor-core kernels: key tiles of 128, at most 16 (+1 for window alignment) tiles per block, and a
+// grid aimed at one wave of the 148 SMs of a B200 when the problem is small enough for that.
+constexpr int kTcTileKeys = 128;
+constexpr int kTcMaxChunkTiles = 16;
+constexpr int kTcTargetBlocks = 148;
+constexpr int kTcMaxWindow = 1024;
+
+// blocks per unit (grid.x) of the tensor-core kernels
+__host__ __device__ inline int tc_chunks_per_unit(int units, int max_seqlen)
+{
+    const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
+    int a = kTcTargetBlocks / units;
+    const int b = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
+    if (a < 1) a = 1;
+    if (a > max_tiles) a = max_tiles;
+    return a > b ? a : b;
+}
+// keys per block when `n_keys` keys are split over `chunks` blocks in whole tiles, rounded up to a
+// multiple of `align` (1 for the statistics sweep, omega for the scoring sweep)
+__host__ __device__ inline int tc_chunk_len(int n_keys, int chunks, int align)
+{
+    const int tiles = (n_keys + kTcTileKeys - 1) / kTcTileKeys;
+    const int ct = (tiles + chunks - 1) / chunks;
+    const int len = ct * kTcTileKeys;
+    return (len + align - 1) / align * align;
+}
+
+// device status bits
+constexpr int kStatusWaitExpired = 1;   // a bounded wait inside a kernel ran out; results are invalid
 
 Workspace plan_workspace(const KShape &ks);
 
@@ -91,6 +124,35 @@ struct LayerTable {
 cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const LayerTable &tab,
                           const int *window_idx, const int *cu_out, int keep_capacity,
                           cudaStream_t stream);
+
+// Eq. 4 for one window of `size` values: mean of the p largest.  Elements are visited in the
+// strict order (value descending, position ascending), so equal values are each taken once.
+__device__ inline float pool_top_p(const float *w, int size, int p)
+{
+    if (p >= size) {
+        float acc = 0.f;
+        for (int x = 0; x < size; ++x) acc += w[x];
+        return acc / (float)size;
+    }
+    float acc = 0.f, prev_v = INFINITY;
+    int prev_i = -1;
+    for (int round = 0; round < p; ++round) {
+        float best_v = -INFINITY;
+        int best_i = size;
+        for (int x = 0; x < size; ++x) {
+            float v = w[x];
+            bool after_prev = v < prev_v || (v == prev_v && x > prev_i);
+            if (after_prev && (v > best_v || best_i == size)) {
+                best_v = v;
+                best_i = x;
+            }
+        }
+        acc += best_v;
+        prev_v = best_v;
+        prev_i = best_i;
+    }
+    return acc / (float)p;
+}
 
 void count_launches(int n);
 void set_error_detail(const char *fmt, ...);

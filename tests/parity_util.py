@@ -54,6 +54,7 @@ def run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_AUTO, staged=False, want_
         binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
                                    out["window_idx"], out["kept_len"], work, keep_capacity=out["keep_capacity"])
     torch.cuda.synchronize()
+    assert binding.device_status(work) == 0, "a kernel reported an expired wait"
     return {
         "prob": prob,
         "window_scores": out["window_scores"].cpu().numpy(),

@@ -13,7 +13,21 @@ import parity_util as pu
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = {"simt": binding.WKV_SCORE_SIMT, "auto": binding.WKV_SCORE_AUTO}
+# "tc" forces the tensor-core (tcgen05) score kernels, "simt" the CUDA-core ones; the full-size
+# configuration tests below use AUTO, which picks the tensor-core kernels for bf16 inputs
+IMPLS = {"simt": binding.WKV_SCORE_SIMT, "tc": binding.WKV_SCORE_TCGEN05, "auto": binding.WKV_SCORE_AUTO}
+
+
+def impl_for(w, impl):
+    """fp32 inputs have no tensor-core path: forcing it must be refused, so those cases run AUTO."""
+    if impl == "tc" and w.dtype == "f32":
+        prob = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05)
+        with pytest.raises(binding.WkvError) as e:
+            binding.wkv_score_windows(prob, torch.zeros(16, device="cuda"), torch.zeros(16, device="cuda"),
+                                      torch.zeros(16, device="cuda"), None, prob.alloc_workspace())
+        assert e.value.status == 7
+        return binding.WKV_SCORE_AUTO
+    return IMPLS[impl]
 
 
 def small(dtype="bf16", **kw):
@@ -26,7 +40,7 @@ def small(dtype="bf16", **kw):
 
 
 # ------------------------------------------------------------------ whole path, small shapes
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "tc"])
 @pytest.mark.parametrize("case", [
     dict(),                                                   # bf16, R = 64, ragged last window
     dict(task=wl.TASK_AGGREGATION, top_p=3),
@@ -37,12 +51,13 @@ def small(dtype="bf16", **kw):
     dict(n_q_heads=6, n_kv_heads=2, l_obs=5, window=7, max_seqlen=999),   # odd sizes: R = 15, omega = 7
     dict(max_seqlen=4096 + 16, window=16, budget_frac=0.12),  # review length a multiple of everything
     dict(dtype="f32", head_dim=64, n_q_heads=4, l_obs=8),     # fp32 inputs
+    dict(window=200, max_seqlen=3000, budget_frac=0.3, n_planted=2),   # a window wider than a key tile
     dict(ragged=True, batch=4, max_seqlen=1500),              # packed layout, n_b in [750, 1500]
     dict(ragged=True, batch=3, max_seqlen=700, task=wl.TASK_AGGREGATION, top_p=2, dtype="f32", head_dim=64),
 ], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()) or "base")
 def test_group_small(case, impl):
     w = small(**case)
-    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=IMPLS[impl])
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=impl_for(w, impl))
     assert max_rel < 1e-4           # far inside the 1e-3 bar; a loose bound here would hide a bug
     for b in range(w.batch):
         for h in range(w.n_kv_heads):
@@ -52,7 +67,7 @@ def test_group_small(case, impl):
                 assert set(planted) <= set(gpu["window_idx"][b, h, :k].tolist())
 
 
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "tc"])
 def test_stage_entry_points_and_token_scores(impl):
     w = small(max_seqlen=1100)
     grp = wl.make_group(w, 0)
@@ -65,6 +80,35 @@ def test_stage_entry_points_and_token_scores(impl):
     t_gpu = gpu["token_scores"][:, :, :n_r].astype(np.float64)
     rel = np.abs(t_gpu - t_ref) / t_ref
     assert rel.max() < 1e-4
+
+
+@pytest.mark.parametrize("impl", ["simt", "tc"])
+def test_token_major_key_layout(impl):
+    # K/V stored [B, N, H_kv, d] (head stride < token stride): another order of tensor-map dimensions
+    w = small(batch=2, max_seqlen=777, window=16, task=wl.TASK_AGGREGATION, top_p=5)
+    grp = wl.make_group(w, 0)
+    ref = oracle.compress_group(grp["q_obs"], grp["k_layers"], grp["v_layers"], fill=pu.fill_pattern(w.dtype),
+                                **pu.oracle_kwargs(w, grp))
+    prob = binding.Problem(dtype=w.dtype, batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                           head_dim=w.head_dim, l_obs=w.l_obs, window=w.window, task=w.task, top_p=w.top_p,
+                           max_seqlen=w.max_seqlen, budgets=grp["budgets"], kv_layout="bnhd",
+                           score_impl=IMPLS[impl])
+    q = binding.to_device(grp["q_obs"])
+    ks = [binding.to_device(np.ascontiguousarray(x.transpose(0, 2, 1, 3))) for x in grp["k_layers"]]
+    vs = [binding.to_device(np.ascontiguousarray(x.transpose(0, 2, 1, 3))) for x in grp["v_layers"]]
+    out = prob.alloc_outputs(len(ks), fill_byte=pu.FILL_BYTE)
+    work = prob.alloc_workspace()
+    binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
+                               out["window_idx"], out["kept_len"], work, keep_capacity=out["keep_capacity"])
+    torch.cuda.synchronize()
+    assert binding.device_status(work) == 0
+    gpu = {"window_scores": out["window_scores"].cpu().numpy(), "window_idx": out["window_idx"].cpu().numpy(),
+           "kept_len": out["kept_len"].cpu().numpy()}
+    pu.check_selection(w, grp, gpu, ref)
+    np.testing.assert_array_equal(gpu["window_idx"], ref["window_idx"])
+    for layer in range(len(ks)):
+        np.testing.assert_array_equal(binding.to_host_bits(out["k_out"][layer]), ref["k_out"][layer])
+        np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][layer]), ref["v_out"][layer])
 
 
 def test_same_result_twice_and_across_entry_points():
@@ -155,7 +199,7 @@ def test_gather_with_given_indices(dtype, d, packed_out):
 
 
 # ------------------------------------------------------------------ degenerate cases
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "tc"])
 @pytest.mark.parametrize("case", [
     dict(budget_frac=None, budget_tokens=10 ** 6),            # budget above n: identity copy
     dict(budget_frac=None, budget_tokens=3),                  # budget below alpha: observation rows only
@@ -167,7 +211,7 @@ def test_gather_with_given_indices(dtype, d, packed_out):
 ], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
 def test_degenerate_sizes(case, impl):
     w = small(n_planted=0, **case)
-    grp, ref, gpu, _ = pu.full_check(w, score_impl=IMPLS[impl])
+    grp, ref, gpu, _ = pu.full_check(w, score_impl=impl_for(w, impl))
     if case.get("budget_tokens") == 10 ** 6:
         n = w.max_seqlen
         assert (gpu["kept_len"] == n).all()
