@@ -113,11 +113,36 @@ size_t wkv_workspace_bytes(const wkv_shape *s);
  *   k_leader       DEVICE  keys of the leader
  *   window_scores  DEVICE  out, float [B, H_kv, wkv_kw_max()] ; entries >= K_w,b are not written
  *   token_scores   DEVICE  out or NULL, float [B, H_kv, max(1, max_seqlen - alpha)] ; t_j of Eq. 2
- *   workspace      DEVICE  scratch of wkv_workspace_bytes() bytes
+ *   workspace      DEVICE  scratch of wkv_workspace_bytes() bytes.  Its first int32 is a status
+ *                  word that the kernels only ever OR into (bit 0: a bounded wait inside a kernel
+ *                  expired, results invalid): zero the workspace once after allocating it and read
+ *                  the word whenever convenient.
  */
 int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader,
                       float *window_scores, float *token_scores,
                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The same stage for callers that cannot allocate device memory (no counterpart in the paper: an
+ * engineering variant).  A serving engine that gave all of HBM to its own cache pool at start-up,
+ * or code running where cudaMalloc is forbidden, has no way to provide the workspace above; here
+ * the scratch is a fixed area of WKV_STATIC_SCRATCH_BYTES inside the library image, which every
+ * GPU that loads the library holds until the process exits.  The function allocates and frees
+ * nothing.
+ *   - Shapes whose wkv_workspace_bytes() exceeds WKV_STATIC_SCRATCH_BYTES are refused with
+ *     WKV_ERR_LIMIT before anything is enqueued.
+ *   - The first call on each device looks up the area's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one area: two calls whose kernels may overlap on the GPU
+ *     (different streams, no dependency) race on it.  Calls on one stream are safe.
+ *   - device_status  DEVICE out or NULL: receives 0, or the error bits a kernel set
+ *     (1 = a bounded wait inside a kernel expired and the scores are invalid).
+ * Other arguments and results exactly as wkv_score_windows.
+ */
+#define WKV_STATIC_SCRATCH_BYTES (4u << 20)
+int wkv_score_windows_static(const wkv_shape *s, const void *q_obs, const void *k_leader,
+                             float *window_scores, float *token_scores, int32_t *device_status,
+                             void *cuda_stream);
 
 /*
  * Budgeted selection (sentence after Eq. 4): per unit the k highest window scores,

@@ -23,7 +23,7 @@ WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max",
-    "wkv_workspace_bytes", "wkv_score_windows", "wkv_select_topk_windows", "wkv_gather_kv",
+    "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
     L.wkv_workspace_bytes.argtypes = [sp]
     L.wkv_score_windows.restype = ctypes.c_int
     L.wkv_score_windows.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp]
+    L.wkv_score_windows_static.restype = ctypes.c_int
+    L.wkv_score_windows_static.argtypes = [sp, vp, vp, vp, vp, vp, vp]
     L.wkv_select_topk_windows.restype = ctypes.c_int
     L.wkv_select_topk_windows.argtypes = [sp, vp, vp, vp, vp]
     L.wkv_gather_kv.restype = ctypes.c_int
@@ -235,6 +237,19 @@ def wkv_score_windows(prob: Problem, q_obs, k_leader, window_scores, token_score
     _check(lib().wkv_score_windows(ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader), _ptr(window_scores),
                                    _ptr(token_scores), _ptr(workspace), workspace.numel(), _stream(stream)),
            "wkv_score_windows")
+
+
+WKV_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def wkv_score_windows_static(prob: Problem, q_obs, k_leader, window_scores, token_scores=None,
+                             device_status=None, stream=None) -> None:
+    """Scoring without a caller workspace: for hosts that may not allocate device memory.  The
+    scratch is a fixed area inside the library (at most WKV_STATIC_SCRATCH_BYTES; larger shapes
+    raise), shared by all calls on the device, so overlapping calls must be serialised."""
+    _check(lib().wkv_score_windows_static(ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader),
+                                          _ptr(window_scores), _ptr(token_scores), _ptr(device_status),
+                                          _stream(stream)), "wkv_score_windows_static")
 
 
 def wkv_select_topk_windows(prob: Problem, window_scores, window_idx, kept_len, stream=None) -> None:

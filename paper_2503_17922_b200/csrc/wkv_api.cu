@@ -53,7 +53,7 @@ static int elem_bytes(int dtype) { return dtype == WKV_F32 ? 4 : 2; }
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Validates the shape and fills the kernel-side copy.  `seqlens` are read from the host arrays.
-static int resolve(const wkv_shape *s, KShape &ks)
+int resolve(const wkv_shape *s, KShape &ks)
 {
     if (!s) {
         set_error_detail("shape is NULL");
@@ -163,7 +163,7 @@ static int resolve(const wkv_shape *s, KShape &ks)
     return WKV_OK;
 }
 
-static int check_cuda(cudaError_t e, const char *what)
+int check_cuda(cudaError_t e, const char *what)
 {
     if (e == cudaSuccess) return WKV_OK;
     set_error_detail("%s: %s", what, cudaGetErrorString(e));
@@ -207,7 +207,7 @@ static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace
     return WKV_OK;
 }
 
-static int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
+int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
                     float *window_scores, float *token_scores, void *workspace, cudaStream_t stream)
 {
     if (!aligned16(q) || !aligned16(k)) {

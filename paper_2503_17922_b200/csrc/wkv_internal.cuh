@@ -154,6 +154,12 @@ __device__ inline float pool_top_p(const float *w, int size, int p)
     return acc / (float)p;
 }
 
+// host side of the boundary, shared by the translation units that export entry points
+int resolve(const wkv_shape *s, KShape &ks);            // validates the shape, fills the kernel-side copy
+int check_cuda(cudaError_t e, const char *what);         // cudaError_t -> wkv_status with detail
+int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
+             float *window_scores, float *token_scores, void *workspace, cudaStream_t stream);
+
 void count_launches(int n);
 void set_error_detail(const char *fmt, ...);
 
