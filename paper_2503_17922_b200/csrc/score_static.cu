@@ -74,12 +74,13 @@ extern "C" int wkv_score_windows_static(const wkv_shape *s, const void *q_obs, c
     st = static_scratch(&scratch);
     if (st != WKV_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    // the status word is the only part of the area that must start from zero; the kernels write
-    // every statistic they later read
-    st = check_cuda(cudaMemsetAsync(static_cast<char *>(scratch) + ws.status_off, 0, sizeof(int), stream),
-                    "clearing the status word");
+    // the status word and the grid-synchronisation words behind it are the only part of the area
+    // that must start from zero; the kernels write every statistic they later read
+    st = check_cuda(cudaMemsetAsync(static_cast<char *>(scratch) + ws.status_off, 0, ws.stats_off - ws.status_off,
+                                    stream),
+                    "clearing the status and synchronisation words");
     if (st != WKV_OK) return st;
-    st = do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, scratch, stream);
+    st = do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, nullptr, nullptr, scratch, stream);
     if (st != WKV_OK) return st;
     if (device_status)
         st = check_cuda(cudaMemcpyAsync(device_status, static_cast<char *>(scratch) + ws.status_off, sizeof(int),

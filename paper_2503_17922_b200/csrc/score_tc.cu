@@ -1,20 +1,31 @@
-// Tensor-core score kernels (tcgen05 + tensor memory + TMA) for bf16 inputs: Eq. 1-4 of the leader.
+// Tensor-core score kernel (tcgen05 + tensor memory + TMA) for bf16 inputs: Eq. 1-4 of the leader
+// and, when asked, the budgeted selection, in ONE cooperative launch.
 //
 // The token score of Eq. 2, t_j = sum_i exp(s_ij) / Z_i, needs every row's softmax normaliser
 // Z_i (a reduction over all keys) before any column sum can be finished, so the keys are swept
-// twice:
-//   score_stats_tc  sweep 1.  D[rows, keys] = Q K^T per 128-key tile with the observation rows on
-//                   the tensor-memory lanes: one thread owns one row and keeps its running
-//                   (max, sum exp2) without any cross-thread traffic (Eq. 1's normaliser, causal
-//                   mask on the tiles that touch the observation window).  K comes from HBM.
-//   score_pool_tc   sweep 2.  D[keys, rows] = K Q^T with the keys on the lanes: one thread owns one
-//                   key and sums exp2(x_ij - lse2_i) over the rows (Eq. 2), the block then pools its
-//                   windows (Eq. 3-4).  K comes from L2 when the leader's keys fit there.
-// Both kernels are warp-specialised: warp 0 issues the TMA tile loads (4-stage ring), warp 1
-// issues the MMAs into a double-buffered accumulator in tensor memory, warps 4-7 and 8-11 are two
-// compute groups that take alternate tiles.  The contraction is the only tensor-core work; the
-// exponentials, sums and the pooling are fp32 on the CUDA cores, in a fixed order.
+// twice, with a grid-wide barrier in between:
+//   sweep 1  D[rows, keys] = Q K^T per 128-key tile with the observation rows on the tensor-memory
+//            lanes: one thread owns one row and keeps its running (max, sum exp2) without any
+//            cross-thread traffic (Eq. 1's normaliser, causal mask on the tiles that touch the
+//            observation window).  K comes from HBM.
+//   sweep 2  D[keys, rows] = K Q^T with the keys on the lanes: one thread owns one key and sums
+//            exp2(x_ij - lse2_i) over the rows (Eq. 2); the block then pools its windows (Eq. 3-4).
+//            The block re-reads the keys it streamed in sweep 1, now from L2.
+//   select   the block that finishes a unit's last windows runs the radix selection for that unit.
+// Units are taken in waves whose keys fit L2 together.  A work item is (unit, chunk of <= 17 key
+// tiles); the persistent blocks (at most one per SM) take the items of a wave round-robin.
+//
+// Warp roles: warp 0 issues the TMA tile loads (4-stage ring), warp 1 issues the MMAs into NG
+// accumulator buffers in tensor memory, and NG compute groups of four warps (one warp per 32-lane
+// quarter of tensor memory) take the tiles round-robin, each with its own buffer, 32 columns at a
+// time; the four warps that share an SM sub-partition cover each other's load latency.  The
+// contraction is the only tensor-core work; exponentials, sums and pooling are fp32 on the CUDA
+// cores in a fixed order, so results are bit-identical from run to run.
+//
+// Every wait is bounded (mbarriers and the grid barrier): on expiry the block sets bit 0 of the
+// status word, drains its own TMA loads, frees its tensor memory and returns.
 #include "tc_common.cuh"
+#include "topk_block.cuh"
 #include "wkv_internal.cuh"
 
 #include <cuda.h>
@@ -27,24 +38,29 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 384;
 constexpr int kStages = 4;
+constexpr int kMaxGroups = 4;
+__host__ __device__ constexpr int groups_for(int mb) { return mb == 1 ? 4 : 2; }
+__host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for(mb) * 128; }
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
 constexpr int kChunkCap = kTcMaxChunkTiles * kTile + kTcMaxWindow;   // token scores a block may hold
+constexpr int kSyncTickets = 16;                         // sync[0] barrier count, sync[1] generation, then tickets
 
 struct TcArgs {
     KShape s;
     float2 *stats;          // [units][n_stat_chunks][r_pad]
     float *window_scores;
     float *token_scores;
+    int *window_idx;        // fused selection when non-null
+    int *kept_len;
     int *status;
+    int *sync;
     int n_stat_chunks, r_pad;
-    int chunks_per_unit;
+    int chunks_per_unit, units_per_wave;
     int kblocks;            // head_dim / 64
     int slot_tok, slot_h, slot_b;   // which tensor-map coordinate (1..3) carries token / head / batch
     int r16;                // observation rows rounded up to a multiple of 16
-    int tmem_cols;          // tensor-memory columns of the scoring kernel
 };
 
 __device__ __forceinline__ uint8_t *align_1024(uint8_t *p)
@@ -53,10 +69,10 @@ __device__ __forceinline__ uint8_t *align_1024(uint8_t *p)
 }
 
 struct Barriers {
-    uint64_t full[kStages];    // TMA -> MMA: the stage holds a key tile
-    uint64_t empty[kStages];   // MMA -> TMA: the MMAs that read the stage have completed
-    uint64_t tfull[2];         // MMA -> compute group: the accumulator buffer is complete
-    uint64_t tempty[2];        // compute group -> MMA: the accumulator buffer has been read
+    uint64_t full[kStages];        // TMA -> MMA: the stage holds a key tile
+    uint64_t empty[kStages];       // MMA -> TMA: the MMAs that read the stage have completed
+    uint64_t tfull[kMaxGroups];    // MMA -> compute group: the accumulator buffer is complete
+    uint64_t tempty[kMaxGroups];   // compute group -> MMA: the accumulator buffer has been read
 };
 
 __device__ __forceinline__ void init_barriers(Barriers &bar)
@@ -65,391 +81,523 @@ __device__ __forceinline__ void init_barriers(Barriers &bar)
         mbar_init(&bar.full[i], 1);
         mbar_init(&bar.empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kMaxGroups; ++i) {
         mbar_init(&bar.tfull[i], 1);
-        mbar_init(&bar.tempty[i], 128);
+        mbar_init(&bar.tempty[i], 4);      // one arrival per warp of the group
     }
     fence_barrier_init();
 }
 
-// Producer loop: key tiles t = 0 .. n_tiles-1 of the block into the stage ring, then waits until the
-// last MMAs have released their stages (so nothing is in flight when the block ends).
-__device__ __forceinline__ void produce_tiles(const CUtensorMap *tmap, const TcArgs &a, Barriers &bar,
-                                              uint8_t *k_stage0, int n_tiles, int tok0, int h, int bcoord,
-                                              volatile int *abort_flag)
+// A compute warp waits through its lane 0 only (fewer threads hammering the barrier word leaves the
+// shared-memory / special-function issue queue to the real work); the result is broadcast.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int lane)
 {
-    const int stage_bytes = a.kblocks * kRegion;
-    tma_prefetch_desc(tmap);
-    int issued = 0;
-    for (int t = 0; t < n_tiles; ++t) {
-        const int st = t % kStages;
-        if (t >= kStages && !mbar_wait(&bar.empty[st], ((t / kStages) - 1) & 1, abort_flag)) break;
-        mbar_arrive_expect_tx(&bar.full[st], (uint32_t)stage_bytes);
-        const int tok = tok0 + t * kTile;
-        const int c1 = a.slot_tok == 1 ? tok : (a.slot_h == 1 ? h : bcoord);
-        const int c2 = a.slot_tok == 2 ? tok : (a.slot_h == 2 ? h : bcoord);
-        const int c3 = a.slot_tok == 3 ? tok : (a.slot_h == 3 ? h : bcoord);
-        for (int kb = 0; kb < a.kblocks; ++kb)
-            tma_load_4d(k_stage0 + st * stage_bytes + kb * kRegion, tmap, &bar.full[st], kb * 64, c1, c2, c3);
-        ++issued;
-    }
-    for (int t = issued > kStages ? issued - kStages : 0; t < issued; ++t) {
-        const int st = t % kStages;
-        if (!mbar_wait(&bar.empty[st], (t / kStages) & 1, abort_flag)) {
-            // giving up: the loads already issued must still land before the block may end
-            volatile int never = 0;
-            mbar_wait(&bar.full[st], (t / kStages) & 1, &never);
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// every lane has finished reading the accumulator buffer: hand it back to the MMA warp
+__device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
+{
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+
+// Grid-wide barrier of a cooperative launch (all blocks resident).  sync[0] counts arrivals and is
+// reset by the last arriver, sync[1] is the generation the others wait on.  Bounded: a block that
+// waits longer than two seconds gives up, sets its abort flag and the caller tears the block down.
+__device__ __forceinline__ int ld_acquire_gpu(const int *p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void grid_barrier(int *sync, int n_blocks, volatile int *abort_flag)
+{
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && !*abort_flag) {
+        const int gen = ld_acquire_gpu(&sync[1]);
+        if (atomicAdd(&sync[0], 1) == n_blocks - 1) {
+            atomicExch(&sync[0], 0);
+            __threadfence();
+            atomicAdd(&sync[1], 1);
+        } else {
+            const unsigned long long t0 = global_timer_ns();
+            while (ld_acquire_gpu(&sync[1]) == gen) {
+                __nanosleep(64);
+                if (global_timer_ns() - t0 > 2 * kWaitLimitNs) {
+                    *abort_flag = 1;
+                    break;
+                }
+            }
         }
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+// geometry of one work item
+struct Item {
+    int unit, chunk, b, h;
+    int n, n_r;
+    long long off;
+    int j_begin, j_end, n_tiles;
+};
+
+// ---------------------------------------------------------------------------------------------
+// per-element work of the two sweeps
+// ---------------------------------------------------------------------------------------------
+// sweep 1: online-softmax update of one row with 32 more logits (raw dot products; c = log2(e)/sqrt(d))
+__device__ __forceinline__ void stats_update(float (&v)[32], bool fast, int jb, int limit, float c, float &m,
+                                             float &l)
+{
+    if (!fast) {
+#pragma unroll
+        for (int x = 0; x < 32; ++x)
+            if (jb + x > limit) v[x] = -INFINITY;
+    }
+    float g0 = fmaxf(v[0], v[1]), g1 = fmaxf(v[2], v[3]);
+#pragma unroll
+    for (int x = 4; x < 32; x += 4) {
+        g0 = fmaxf(g0, fmaxf(v[x], v[x + 1]));
+        g1 = fmaxf(g1, fmaxf(v[x + 2], v[x + 3]));
+    }
+    const float m_new = fmaxf(m, fmaxf(g0, g1));
+    if (m_new > -INFINITY) {
+        const float mc = m_new * c;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int x = 0; x < 32; x += 4) {
+            a0 += fast_exp2(fmaf(v[x], c, -mc));
+            a1 += fast_exp2(fmaf(v[x + 1], c, -mc));
+            a2 += fast_exp2(fmaf(v[x + 2], c, -mc));
+            a3 += fast_exp2(fmaf(v[x + 3], c, -mc));
+        }
+        const float add = (a0 + a1) + (a2 + a3);
+        l = m_new == m ? l + add : l * fast_exp2((m - m_new) * c) + add;
+        m = m_new;
+    }
+}
+// sweep 2: adds exp2(x*c - lse2) of 32 (or 16) rows to the four partial sums of a key
+template <int N>
+__device__ __forceinline__ void score_accumulate(const float (&v)[N], const float *nl_base, float c, float &a0,
+                                                 float &a1, float &a2, float &a3)
+{
+#pragma unroll
+    for (int x = 0; x < N; x += 4) {
+        const float4 nl = *reinterpret_cast<const float4 *>(nl_base + x);
+        a0 += fast_exp2(fmaf(v[x], c, nl.x));
+        a1 += fast_exp2(fmaf(v[x + 1], c, nl.y));
+        a2 += fast_exp2(fmaf(v[x + 2], c, nl.z));
+        a3 += fast_exp2(fmaf(v[x + 3], c, nl.w));
+    }
+}
+
+// Eq. 4 for windows whose length omega is a power of two <= 32: a warp takes 32/omega windows at a
+// time, one lane per token.  The rank of a token inside its window (value descending, position
+// ascending) comes from omega shuffles; the p best are summed by a butterfly in a fixed order.
+__device__ __forceinline__ void pool_windows_warp(const float *t_chunk, int n_tok, int omega, int p, float *out,
+                                                  int warp, int n_warps, int lane)
+{
+    const int per_warp = 32 / omega;
+    const int n_win = (n_tok + omega - 1) / omega;
+    const int e = lane % omega, sub = lane / omega;
+    for (int w0 = warp * per_warp; w0 < n_win; w0 += n_warps * per_warp) {
+        const int w = w0 + sub;
+        const int j = w * omega + e;
+        const bool valid = w < n_win && j < n_tok;
+        const float v = valid ? t_chunk[j] : -INFINITY;
+        int rank = 0;
+        for (int x = 0; x < omega; ++x) {
+            const float o = __shfl_sync(0xffffffffu, v, sub * omega + x);
+            rank += (o > v || (o == v && x < e)) ? 1 : 0;
+        }
+        const int size = w < n_win ? min(omega, n_tok - w * omega) : 1;
+        const int p_eff = p < size ? p : size;
+        float acc = (valid && rank < p_eff) ? v : 0.f;
+        for (int o = 1; o < omega; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (e == 0 && w < n_win) out[w] = acc / (float)p_eff;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// sweep 1: per-row partial (max, sum exp2) over the block's keys
+// the kernel
 // ---------------------------------------------------------------------------------------------
 template <int MB>   // 128-row blocks of observation rows: 1 (R <= 128) or 2 (R <= 256)
-__global__ void __launch_bounds__(kThreads, 1)
-score_stats_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ TcArgs a,
-               const __nv_bfloat16 *__restrict__ q)
+// 18 warps put five on one SM sub-partition (16K registers): 96 registers per thread at most
+__global__ void __launch_bounds__(block_threads(MB), 1)
+score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ TcArgs a,
+                 const __nv_bfloat16 *__restrict__ q)
 {
+    constexpr int NG = groups_for(MB);
+    constexpr int kThreads = block_threads(MB);
+    constexpr int q_rows = MB * 128;
+    constexpr int q_region = q_rows * 128;                // bytes of one 64-column block of the Q image
+    constexpr uint32_t buf_cols = MB * 128;               // accumulator buffer stride in tensor memory
+    constexpr uint32_t tmem_cols = 512;
+    static_assert(NG * buf_cols <= tmem_cols, "accumulator buffers exceed tensor memory");
+
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) Barriers bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ float2 part[2][MB][128];
+    __shared__ int flag_s;
+    __shared__ float2 part[NG][MB][128];
+    __shared__ __align__(16) float neg_lse2[256];        // -log2 of the row normaliser; -inf for padding rows
+    __shared__ float t_chunk[kChunkCap];
+    __shared__ TopkSmem topk_sm;
 
     const KShape &s = a.s;
-    const int unit = blockIdx.y, chunk = blockIdx.x;
-    const int b = unit / s.hkv, h = unit % s.hkv;
-    const SeqInfo si = seq_info(s, b);
-    const int n = si.n, n_r = n - s.alpha;
-    float2 *out = a.stats + ((size_t)unit * a.n_stat_chunks + chunk) * a.r_pad;
-    const int len = tc_chunk_len(n, a.chunks_per_unit, 1);
-    const int j_begin = chunk * len;
-    if (n_r <= 0 || j_begin >= n) {
-        for (int r = threadIdx.x; r < a.r_pad; r += kThreads) out[r] = make_float2(-INFINITY, 0.f);
-        return;
-    }
-    const int j_end = min(n, j_begin + len);
-    const int n_tiles = (j_end - j_begin + kTile - 1) / kTile;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int units = s.batch * s.hkv;
+    const int cpu = a.chunks_per_unit;
+    const float c = s.scale_log2;
 
     uint8_t *q_img = align_1024(smem_raw);
-    constexpr int q_rows = MB * 128;
-    constexpr int q_region = q_rows * 128;
     uint8_t *k_stage0 = q_img + a.kblocks * q_region;
     const int stage_bytes = a.kblocks * kRegion;
-    constexpr uint32_t tmem_cols = MB * 256;    // two accumulator buffers of MB x 128 columns
+    const int ksteps = s.d / 16;
 
     if (threadIdx.x == 0) {
         init_barriers(bar);
         abort_s = 0;
     }
     if (warp == 1) tmem_alloc(&tmem_base_s, tmem_cols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_s;
+    if (warp == 0 && lane == 0) tma_prefetch_desc(&tmap);
 
-    // Q image: row r of the image is observation row (r mod Rp); with Rp < 128 the rows repeat so
-    // that all 128 lanes work, each copy taking its own slice of a tile's columns
+    // Row layout of the Q image: image row r holds observation row (r mod Rp); with Rp < 128 the rows
+    // repeat so that all 128 lanes work in sweep 1, each copy taking its own slice of a tile's columns.
+    // Rows [0, r16) of the image are the B operand of sweep 2.
     const int Rp = MB == 2 ? 256 : (s.R <= 32 ? 32 : (s.R <= 64 ? 64 : 128));
-    const __nv_bfloat16 *q_unit = q + b * s.qsb + (long long)h * s.G * s.qsh;
-    const int vec_per_row = s.d / 8;
-    for (int idx = threadIdx.x; idx < q_rows * vec_per_row; idx += kThreads) {
-        const int r = idx / vec_per_row, cc = idx % vec_per_row;
-        const int rq = r % Rp;
-        int4 v = make_int4(0, 0, 0, 0);
-        if (rq < s.R) {
-            const int g = rq / s.alpha, i = rq % s.alpha;
-            v = *reinterpret_cast<const int4 *>(q_unit + g * s.qsh + i * s.qst + cc * 8);
-        }
-        *reinterpret_cast<int4 *>(q_img + (cc >> 3) * q_region + swz128_offset(r, cc & 7)) = v;
-    }
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = tmem_base_s;
+    int q_unit_loaded = -1;
+    uint32_t it = 0;            // key tiles this block has pushed through the pipeline so far
+    uint32_t p_issued = 0;      // producer thread only: tiles whose loads have been issued
 
-    if (warp == 0) {
-        if (lane == 0)
-            produce_tiles(&tmap, a, bar, k_stage0, n_tiles, (int)si.off + j_begin, h, s.cu ? 0 : b, &abort_s);
-    } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, kTile);
-            const uint32_t q_addr = smem_u32(q_img);
-            const int ksteps = s.d / 16;
-            for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kStages, buf = t & 1;
-                if (!mbar_wait(&bar.full[st], (t / kStages) & 1, &abort_s)) break;
-                if (t >= 2 && !mbar_wait(&bar.tempty[buf], ((t >> 1) - 1) & 1, &abort_s)) break;
-                tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(k_stage0 + st * stage_bytes);
-#pragma unroll
-                for (int mb = 0; mb < MB; ++mb) {
-                    const uint32_t d_tmem = tmem_base + buf * (MB * 128) + mb * 128;
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint32_t kb = ks >> 2, sub = (ks & 3) * 32;
-                        umma_bf16(d_tmem, umma_desc_sw128(q_addr + kb * q_region + mb * kRegion + sub),
-                                  umma_desc_sw128(k_addr + kb * kRegion + sub), idesc, ks > 0);
-                    }
-                }
-                umma_commit(&bar.empty[st]);
-                umma_commit(&bar.tfull[buf]);
+    auto make_item = [&](int unit, int chunk, int review_only, Item &im) {
+        im.unit = unit;
+        im.chunk = chunk;
+        im.b = unit / s.hkv;
+        im.h = unit % s.hkv;
+        const SeqInfo si = seq_info(s, im.b);
+        im.n = si.n;
+        im.n_r = si.n - s.alpha;
+        im.off = si.off;
+        const int n_keys = review_only ? im.n_r : im.n;
+        const int len = tc_chunk_len(n_keys > 0 ? n_keys : 1, cpu, review_only ? s.omega : 1);
+        im.j_begin = chunk * len;
+        im.j_end = min(n_keys, im.j_begin + len);
+        im.n_tiles = im.j_end > im.j_begin ? (im.j_end - im.j_begin + kTile - 1) / kTile : 0;
+    };
+
+    auto load_q_image = [&](const Item &im) {
+        if (q_unit_loaded == im.unit) return;
+        q_unit_loaded = im.unit;
+        const __nv_bfloat16 *q_unit = q + im.b * s.qsb + (long long)im.h * s.G * s.qsh;
+        const int vec_per_row = s.d / 8;
+        for (int idx = threadIdx.x; idx < q_rows * vec_per_row; idx += kThreads) {
+            const int r = idx / vec_per_row, cc = idx % vec_per_row;
+            const int rq = r % Rp;
+            int4 v = make_int4(0, 0, 0, 0);
+            if (rq < s.R) {
+                const int g = rq / s.alpha, i = rq % s.alpha;
+                v = *reinterpret_cast<const int4 *>(q_unit + g * s.qsh + i * s.qst + cc * 8);
             }
+            *reinterpret_cast<int4 *>(q_img + (cc >> 3) * q_region + swz128_offset(r, cc & 7)) = v;
         }
-    } else if (warp >= 4) {
-        const int grp = (warp - 4) >> 2, quarter = warp & 3;
-        const int L = quarter * 32 + lane;
-        const int ncols = MB == 2 ? kTile : Rp;             // columns of a tile this thread reduces
-        const int col0 = MB == 2 ? 0 : (L / Rp) * Rp;       // warp-uniform: Rp is a multiple of 32
-        const float c = s.scale_log2;
-        float m[MB], l[MB];
-        int limit[MB];                                      // last key the row may attend to
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-            m[mb] = -INFINITY;
-            l[mb] = 0.f;
-            const int row = MB == 2 ? mb * 128 + L : L % Rp;
-            limit[mb] = row < s.R ? min(n_r + row % s.alpha, j_end - 1) : -1;
+        fence_proxy_async_smem();
+    };
+
+    // producer: the item's key tiles into the stage ring (the block-wide tile counter `it` keeps the phases)
+    auto produce = [&](const Item &im) {
+        const int tok0 = (int)im.off + im.j_begin;
+        const int bcoord = s.cu ? 0 : im.b;
+        for (int t = 0; t < im.n_tiles; ++t) {
+            const uint32_t g = it + t;
+            const int st = g % kStages;
+            if (g >= kStages && !mbar_wait(&bar.empty[st], ((g / kStages) - 1) & 1, &abort_s)) return;
+            mbar_arrive_expect_tx(&bar.full[st], (uint32_t)stage_bytes);
+            const int tok = tok0 + t * kTile;
+            const int c1 = a.slot_tok == 1 ? tok : (a.slot_h == 1 ? im.h : bcoord);
+            const int c2 = a.slot_tok == 2 ? tok : (a.slot_h == 2 ? im.h : bcoord);
+            const int c3 = a.slot_tok == 3 ? tok : (a.slot_h == 3 ? im.h : bcoord);
+            for (int kb = 0; kb < a.kblocks; ++kb)
+                tma_load_4d(k_stage0 + st * stage_bytes + kb * kRegion, &tmap, &bar.full[st], kb * 64, c1, c2, c3);
+            ++p_issued;
         }
-        for (int t = grp; t < n_tiles; t += 2) {
-            bool ok = mbar_wait(&bar.tfull[grp], (t >> 1) & 1, &abort_s);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+    };
+
+    // MMA issue for one item.  sweep 1: D[rows, keys] = Q K^T (MB row blocks); sweep 2: D[keys, rows] = K Q^T
+    auto issue_mma = [&](const Item &im, bool sweep2) {
+        const uint32_t q_addr = smem_u32(q_img);
+        const uint32_t idesc = sweep2 ? umma_idesc_bf16(128, a.r16) : umma_idesc_bf16(128, kTile);
+        for (int t = 0; t < im.n_tiles; ++t) {
+            const uint32_t g = it + t;
+            const int st = g % kStages, buf = g % NG;
+            if (!mbar_wait(&bar.full[st], (g / kStages) & 1, &abort_s)) return;
+            if (g >= NG && !mbar_wait(&bar.tempty[buf], ((g / NG) - 1) & 1, &abort_s)) return;
             tc_fence_after_sync();
-            const int j0 = j_begin + t * kTile;
-            const bool fast = (j0 + kTile - 1 <= n_r) && (j0 + kTile - 1 < j_end);   // no masking needed
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + grp * (MB * 128) + mb * 128 + col0;
-                for (int cg = 0; cg < ncols; cg += 32) {
-                    float v[32];
-                    tmem_ld32(taddr + cg, v);
-                    if (!fast) {
-                        const int jb = j0 + col0 + cg;
-#pragma unroll
-                        for (int x = 0; x < 32; ++x)
-                            if (jb + x > limit[mb]) v[x] = -INFINITY;
-                    }
-                    float g0 = fmaxf(v[0], v[1]), g1 = fmaxf(v[2], v[3]);
-#pragma unroll
-                    for (int x = 4; x < 32; x += 4) {
-                        g0 = fmaxf(g0, fmaxf(v[x], v[x + 1]));
-                        g1 = fmaxf(g1, fmaxf(v[x + 2], v[x + 3]));
-                    }
-                    const float m_new = fmaxf(m[mb], fmaxf(g0, g1));
-                    if (m_new > -INFINITY) {
-                        const float mc = m_new * c;
-                        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                        for (int x = 0; x < 32; x += 4) {
-                            a0 += fast_exp2(fmaf(v[x], c, -mc));
-                            a1 += fast_exp2(fmaf(v[x + 1], c, -mc));
-                            a2 += fast_exp2(fmaf(v[x + 2], c, -mc));
-                            a3 += fast_exp2(fmaf(v[x + 3], c, -mc));
-                        }
-                        l[mb] = l[mb] * fast_exp2((m[mb] - m_new) * c) + ((a0 + a1) + (a2 + a3));
-                        m[mb] = m_new;
-                    }
-                }
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&bar.tempty[grp]);
-        }
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) part[grp][mb][L] = make_float2(m[mb], l[mb]);
-    }
-
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    if (!abort_s) {
-        // combine the two compute groups and the column slices of each row, in a fixed order
-        const float c = s.scale_log2;
-        const int copies = MB == 2 ? 1 : 128 / Rp;
-        for (int r = threadIdx.x; r < a.r_pad; r += kThreads) {
-            float2 res = make_float2(-INFINITY, 0.f);
-            if (r < s.R) {
-                const int mb = MB == 2 ? r >> 7 : 0, base = MB == 2 ? (r & 127) : r;
-                float M = -INFINITY;
-                for (int g = 0; g < 2; ++g)
-                    for (int cp = 0; cp < copies; ++cp) M = fmaxf(M, part[g][mb][base + cp * Rp].x);
-                float sum = 0.f;
-                for (int g = 0; g < 2; ++g)
-                    for (int cp = 0; cp < copies; ++cp) {
-                        const float2 p = part[g][mb][base + cp * Rp];
-                        if (p.y > 0.f) sum += p.y * exp2f((p.x - M) * c);
-                    }
-                res = make_float2(M * c, sum);
-            }
-            out[r] = res;
-        }
-    } else if (threadIdx.x == 0) {
-        atomicOr(a.status, kStatusWaitExpired);
-    }
-    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
-}
-
-// ---------------------------------------------------------------------------------------------
-// sweep 2: token scores (Eq. 2) and window pooling (Eq. 3-4)
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 1)
-score_pool_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ TcArgs a,
-              const __nv_bfloat16 *__restrict__ q)
-{
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) Barriers bar;
-    __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s;
-    __shared__ __align__(16) float neg_lse2[256];     // -log2 of the row normaliser; -inf for padding rows
-    __shared__ float t_chunk[kChunkCap];
-
-    const KShape &s = a.s;
-    const int unit = blockIdx.y, chunk = blockIdx.x;
-    const int b = unit / s.hkv, h = unit % s.hkv;
-    const SeqInfo si = seq_info(s, b);
-    const int n = si.n, n_r = n - s.alpha;
-    if (n_r <= 0) return;
-    const int len = tc_chunk_len(n_r, a.chunks_per_unit, s.omega);
-    const int j_begin = chunk * len;
-    if (j_begin >= n_r) return;
-    const int j_end = min(n_r, j_begin + len);
-    const int n_tiles = (j_end - j_begin + kTile - 1) / kTile;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    uint8_t *q_img = align_1024(smem_raw);
-    const int q_region = a.r16 * 128;
-    uint8_t *k_stage0 = align_1024(q_img + a.kblocks * q_region);
-    const int stage_bytes = a.kblocks * kRegion;
-    const int buf_cols = a.tmem_cols >> 1;
-
-    if (threadIdx.x == 0) {
-        init_barriers(bar);
-        abort_s = 0;
-    }
-    if (warp == 1) tmem_alloc(&tmem_base_s, (uint32_t)a.tmem_cols);
-
-    const __nv_bfloat16 *q_unit = q + b * s.qsb + (long long)h * s.G * s.qsh;
-    const int vec_per_row = s.d / 8;
-    for (int idx = threadIdx.x; idx < a.r16 * vec_per_row; idx += kThreads) {
-        const int r = idx / vec_per_row, cc = idx % vec_per_row;
-        int4 v = make_int4(0, 0, 0, 0);
-        if (r < s.R) {
-            const int g = r / s.alpha, i = r % s.alpha;
-            v = *reinterpret_cast<const int4 *>(q_unit + g * s.qsh + i * s.qst + cc * 8);
-        }
-        *reinterpret_cast<int4 *>(q_img + (cc >> 3) * q_region + swz128_offset(r, cc & 7)) = v;
-    }
-    // Eq. 1's normaliser of every row from the partial statistics of sweep 1
-    {
-        const int len1 = tc_chunk_len(n, a.chunks_per_unit, 1);
-        const int used = (n + len1 - 1) / len1;
-        for (int r = threadIdx.x; r < 256; r += kThreads) {
-            float v = -INFINITY;
-            if (r < s.R) {
-                const float2 *st = a.stats + (size_t)unit * a.n_stat_chunks * a.r_pad + r;
-                float M = -INFINITY;
-                for (int cidx = 0; cidx < used; ++cidx) M = fmaxf(M, st[(size_t)cidx * a.r_pad].x);
-                float sum = 0.f;
-                for (int cidx = 0; cidx < used; ++cidx) {
-                    const float2 p = st[(size_t)cidx * a.r_pad];
-                    if (p.y > 0.f) sum += p.y * exp2f(p.x - M);
-                }
-                if (sum > 0.f) v = -(M + log2f(sum));
-            }
-            neg_lse2[r] = v;
-        }
-    }
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = tmem_base_s;
-
-    if (warp == 0) {
-        if (lane == 0)
-            produce_tiles(&tmap, a, bar, k_stage0, n_tiles, (int)si.off + j_begin, h, s.cu ? 0 : b, &abort_s);
-    } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(128, a.r16);
-            const uint32_t q_addr = smem_u32(q_img);
-            const int ksteps = s.d / 16;
-            for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kStages, buf = t & 1;
-                if (!mbar_wait(&bar.full[st], (t / kStages) & 1, &abort_s)) break;
-                if (t >= 2 && !mbar_wait(&bar.tempty[buf], ((t >> 1) - 1) & 1, &abort_s)) break;
-                tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(k_stage0 + st * stage_bytes);
-                const uint32_t d_tmem = tmem_base + buf * buf_cols;
+            const uint32_t k_addr = smem_u32(k_stage0 + st * stage_bytes);
+            const uint32_t d_tmem = tmem_base + buf * buf_cols;
+            if (sweep2) {
                 for (int ks = 0; ks < ksteps; ++ks) {
                     const uint32_t kb = ks >> 2, sub = (ks & 3) * 32;
                     umma_bf16(d_tmem, umma_desc_sw128(k_addr + kb * kRegion + sub),
                               umma_desc_sw128(q_addr + kb * q_region + sub), idesc, ks > 0);
                 }
-                umma_commit(&bar.empty[st]);
-                umma_commit(&bar.tfull[buf]);
+            } else {
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb)
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        const uint32_t kb = ks >> 2, sub = (ks & 3) * 32;
+                        umma_bf16(d_tmem + mb * 128, umma_desc_sw128(q_addr + kb * q_region + mb * kRegion + sub),
+                                  umma_desc_sw128(k_addr + kb * kRegion + sub), idesc, ks > 0);
+                    }
+            }
+            umma_commit(&bar.empty[st]);
+            umma_commit(&bar.tfull[buf]);
+        }
+    };
+
+    const int grp = warp >= 2 ? (warp - 2) >> 2 : 0, quarter = warp & 3;
+    const int L = quarter * 32 + lane;
+    const uint32_t taddr_grp = tmem_base + ((uint32_t)(quarter * 32) << 16) + grp * buf_cols;
+
+    // sweep-1 compute: the row's partial (max, sum exp2) over the item's keys -> part[grp][.][L]
+    auto compute_stats = [&](const Item &im) {
+        const int ncols = MB == 2 ? kTile : Rp;             // columns of a tile this thread reduces
+        const int col0 = MB == 2 ? 0 : (L / Rp) * Rp;       // warp-uniform: Rp is a multiple of 32
+        const int gshift = ncols == 128 ? 2 : (ncols == 64 ? 1 : 0);   // log2(32-column groups per row block)
+        const int gmask = (1 << gshift) - 1;
+        const int nslot = MB << gshift;
+        float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+        int limit0, limit1 = -1;                            // last key each row may attend to
+        {
+            const int row = MB == 2 ? L : L % Rp;
+            limit0 = row < s.R ? min(im.n_r + row % s.alpha, im.j_end - 1) : -1;
+            if (MB == 2) limit1 = 128 + L < s.R ? min(im.n_r + (128 + L) % s.alpha, im.j_end - 1) : -1;
+        }
+        const uint32_t taddr = taddr_grp + col0;
+        for (int t = 0; t < im.n_tiles; ++t) {
+            const uint32_t g = it + t;
+            if ((int)(g % NG) != grp) continue;
+            if (!warp_wait(&bar.tfull[grp], (g / NG) & 1, &abort_s, lane)) break;
+            tc_fence_after_sync();
+            const int tile0 = im.j_begin + t * kTile;
+            const int j0 = tile0 + col0;
+            const bool fast = (tile0 + kTile - 1 <= im.n_r) && (tile0 + kTile - 1 < im.j_end);   // no masking
+            // slot sl = 32 columns: row block sl >> gshift, column group sl & gmask
+            for (int sl = 0; sl < nslot; ++sl) {
+                float v[32];
+                tmem_ld32(taddr + (sl >> gshift) * 128 + (sl & gmask) * 32, v);
+                if (sl + 1 == nslot) warp_release(&bar.tempty[grp], lane);   // the buffer may be overwritten now
+                if (MB == 2 && (sl >> gshift)) stats_update(v, fast, j0 + (sl & gmask) * 32, limit1, c, m1, l1);
+                else stats_update(v, fast, j0 + (sl & gmask) * 32, limit0, c, m0, l0);
             }
         }
-    } else if (warp >= 4) {
-        const int grp = (warp - 4) >> 2, quarter = warp & 3;
-        const int L = quarter * 32 + lane;
-        const float c = s.scale_log2;
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + grp * buf_cols;
-        for (int t = grp; t < n_tiles; t += 2) {
-            bool ok = mbar_wait(&bar.tfull[grp], (t >> 1) & 1, &abort_s);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        part[grp][0][L] = make_float2(m0, l0);
+        if (MB == 2) part[grp][MB - 1][L] = make_float2(m1, l1);
+    };
+
+    // sweep-2 compute: token score of key L of every tile of the item -> t_chunk (and token_scores)
+    auto compute_scores = [&](const Item &im) {
+        const int n32 = a.r16 >> 5;                  // 32-row groups; a 16-row tail follows if r16 & 16
+        const bool tail = (a.r16 & 16) != 0;
+        for (int t = 0; t < im.n_tiles; ++t) {
+            const uint32_t g = it + t;
+            if ((int)(g % NG) != grp) continue;
+            if (!warp_wait(&bar.tfull[grp], (g / NG) & 1, &abort_s, lane)) break;
             tc_fence_after_sync();
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            int cg = 0;
-            for (; cg + 32 <= a.r16; cg += 32) {
+            for (int sl = 0; sl < n32; ++sl) {
                 float v[32];
-                tmem_ld32(taddr + cg, v);
-#pragma unroll
-                for (int x = 0; x < 32; x += 4) {
-                    const float4 nl = *reinterpret_cast<const float4 *>(&neg_lse2[cg + x]);
-                    a0 += fast_exp2(fmaf(v[x], c, nl.x));
-                    a1 += fast_exp2(fmaf(v[x + 1], c, nl.y));
-                    a2 += fast_exp2(fmaf(v[x + 2], c, nl.z));
-                    a3 += fast_exp2(fmaf(v[x + 3], c, nl.w));
-                }
+                tmem_ld32(taddr_grp + sl * 32, v);
+                if (sl + 1 == n32 && !tail) warp_release(&bar.tempty[grp], lane);   // the buffer may be overwritten now
+                score_accumulate<32>(v, neg_lse2 + sl * 32, c, a0, a1, a2, a3);
             }
-            if (cg < a.r16) {
-                float v[16];
-                tmem_ld16(taddr + cg, v);
-#pragma unroll
-                for (int x = 0; x < 16; x += 4) {
-                    const float4 nl = *reinterpret_cast<const float4 *>(&neg_lse2[cg + x]);
-                    a0 += fast_exp2(fmaf(v[x], c, nl.x));
-                    a1 += fast_exp2(fmaf(v[x + 1], c, nl.y));
-                    a2 += fast_exp2(fmaf(v[x + 2], c, nl.z));
-                    a3 += fast_exp2(fmaf(v[x + 3], c, nl.w));
-                }
+            if (tail) {
+                float vt[16];
+                tmem_ld16(taddr_grp + n32 * 32, vt);
+                warp_release(&bar.tempty[grp], lane);
+                score_accumulate<16>(vt, neg_lse2 + n32 * 32, c, a0, a1, a2, a3);
             }
-            tc_fence_before_sync();
-            mbar_arrive(&bar.tempty[grp]);
             const float tj = (a0 + a1) + (a2 + a3);
-            const int j = j_begin + t * kTile + L;
-            if (j < j_end) {
-                t_chunk[j - j_begin] = tj;
-                if (a.token_scores) a.token_scores[(size_t)unit * s.nr_max + j] = tj;
+            const int j = im.j_begin + t * kTile + L;
+            if (j < im.j_end) {
+                t_chunk[j - im.j_begin] = tj;
+                if (a.token_scores) a.token_scores[(size_t)im.unit * s.nr_max + j] = tj;
             }
+        }
+    };
+
+    const int n_waves = (units + a.units_per_wave - 1) / a.units_per_wave;
+    for (int wave = 0; wave < n_waves && !abort_s; ++wave) {
+        const int u0 = wave * a.units_per_wave;
+        const int nu = min(a.units_per_wave, units - u0);
+        const int n_items = nu * cpu;
+
+        // ------------------------------------------------------------------ sweep 1
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            Item im;
+            make_item(u0 + item / cpu, item % cpu, 0, im);
+            float2 *out = a.stats + ((size_t)im.unit * a.n_stat_chunks + im.chunk) * a.r_pad;
+            if (im.n_r <= 0 || im.n_tiles == 0) {
+                for (int r = threadIdx.x; r < a.r_pad; r += kThreads) out[r] = make_float2(-INFINITY, 0.f);
+                continue;
+            }
+            load_q_image(im);
+            __syncthreads();
+            if (warp == 0) {
+                if (lane == 0) produce(im);
+            } else if (warp == 1) {
+                if (lane == 0) issue_mma(im, false);
+            } else {
+                compute_stats(im);
+            }
+            it += im.n_tiles;
+            tc_fence_before_sync();
+            __syncthreads();
+            tc_fence_after_sync();
+            if (abort_s) break;
+            // combine the compute groups and the column slices of each row, in a fixed order
+            const int copies = MB == 2 ? 1 : 128 / Rp;
+            for (int r = threadIdx.x; r < a.r_pad; r += kThreads) {
+                float2 res = make_float2(-INFINITY, 0.f);
+                if (r < s.R) {
+                    const int mb = MB == 2 ? r >> 7 : 0, base = MB == 2 ? (r & 127) : r;
+                    float M = -INFINITY;
+                    for (int g = 0; g < NG; ++g)
+                        for (int cp = 0; cp < copies; ++cp) M = fmaxf(M, part[g][mb][base + cp * Rp].x);
+                    float sum = 0.f;
+                    for (int g = 0; g < NG; ++g)
+                        for (int cp = 0; cp < copies; ++cp) {
+                            const float2 p = part[g][mb][base + cp * Rp];
+                            if (p.y > 0.f) sum += p.y * exp2f((p.x - M) * c);
+                        }
+                    res = make_float2(M * c, sum);
+                }
+                out[r] = res;
+            }
+        }
+
+        grid_barrier(a.sync, gridDim.x, &abort_s);
+        if (abort_s) break;
+
+        // ------------------------------------------------------------------ sweep 2 (+ selection)
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            Item im;
+            make_item(u0 + item / cpu, item % cpu, 1, im);
+            const int kw = num_windows(im.n, s.alpha, s.omega);
+            if (im.n_r <= 0 || im.n_tiles == 0) {
+                // a unit without review context still gets its (empty) selection, from its first item
+                if (a.window_idx && im.n_r <= 0 && im.chunk == 0) {
+                    select_topk_block<kThreads>(topk_sm, a.window_scores + (size_t)im.unit * s.kw_max, 0, 0, s.k_max,
+                                                a.window_idx + (size_t)im.unit * s.k_max, a.kept_len + im.unit,
+                                                im.n, s.alpha, s.omega);
+                    __syncthreads();
+                }
+                continue;
+            }
+            load_q_image(im);
+            {
+                // Eq. 1's normaliser of every row: merge the partial statistics of the unit's chunks
+                const int len1 = tc_chunk_len(im.n, cpu, 1);
+                const int used = (im.n + len1 - 1) / len1;
+                for (int r = threadIdx.x; r < 256; r += kThreads) {
+                    float v = -INFINITY;
+                    if (r < s.R) {
+                        const float2 *st = a.stats + (size_t)im.unit * a.n_stat_chunks * a.r_pad + r;
+                        float M = -INFINITY, sum = 0.f;
+#pragma unroll 6
+                        for (int cidx = 0; cidx < used; ++cidx) {
+                            const float2 p = __ldcg(st + (size_t)cidx * a.r_pad);
+                            if (p.y > 0.f) {
+                                const float Mn = fmaxf(M, p.x);
+                                sum = sum * exp2f(M - Mn) + p.y * exp2f(p.x - Mn);
+                                M = Mn;
+                            }
+                        }
+                        if (sum > 0.f) v = -(M + log2f(sum));
+                    }
+                    neg_lse2[r] = v;
+                }
+            }
+            __syncthreads();
+            if (warp == 0) {
+                if (lane == 0) produce(im);
+            } else if (warp == 1) {
+                if (lane == 0) issue_mma(im, true);
+            } else {
+                compute_scores(im);
+            }
+            it += im.n_tiles;
+            tc_fence_before_sync();
+            __syncthreads();
+            tc_fence_after_sync();
+            if (abort_s) break;
+            // Eq. 3-4: the item's windows (its first key is a multiple of omega)
+            {
+                const int n_tok = im.j_end - im.j_begin;
+                float *ws_out = a.window_scores + (size_t)im.unit * s.kw_max + im.j_begin / s.omega;
+                if (s.omega <= 32 && (s.omega & (s.omega - 1)) == 0) {
+                    pool_windows_warp(t_chunk, n_tok, s.omega, s.p, ws_out, warp, kThreads / 32, lane);
+                } else {
+                    const int n_win = (n_tok + s.omega - 1) / s.omega;
+                    for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
+                        const int lo = lw * s.omega;
+                        ws_out[lw] = pool_top_p(t_chunk + lo, min(s.omega, n_tok - lo), s.p);
+                    }
+                }
+            }
+            if (a.window_idx) {
+                // the block that completes the unit's last windows selects for the unit
+                const int len2 = tc_chunk_len(im.n_r, cpu, s.omega);
+                const int used2 = (im.n_r + len2 - 1) / len2;
+                __threadfence();
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    int *ticket = a.sync + kSyncTickets + im.unit;
+                    const int last = atomicAdd(ticket, 1) == used2 - 1;
+                    if (last) atomicExch(ticket, 0);
+                    __threadfence();
+                    flag_s = last;
+                }
+                __syncthreads();
+                if (flag_s) {
+                    const SeqInfo si = seq_info(s, im.b);
+                    select_topk_block<kThreads>(topk_sm, a.window_scores + (size_t)im.unit * s.kw_max, kw,
+                                                num_selected(im.n, s.alpha, s.omega, si.budget), s.k_max,
+                                                a.window_idx + (size_t)im.unit * s.k_max, a.kept_len + im.unit,
+                                                im.n, s.alpha, s.omega);
+                }
+            }
+            __syncthreads();   // t_chunk, neg_lse2 and the selection scratch are reused by the next item
         }
     }
 
+    // ------------------------------------------------------------------ teardown
+    __syncthreads();
+    if (warp == 0 && lane == 0) {
+        // nothing of this block may be in flight when it ends: the last MMAs must have released
+        // their stages; after a failed wait, the loads already issued must still land
+        for (uint32_t g = p_issued > kStages ? p_issued - kStages : 0; g < p_issued; ++g) {
+            const int st = g % kStages;
+            if (!mbar_wait(&bar.empty[st], (g / kStages) & 1, &abort_s)) {
+                volatile int never = 0;
+                mbar_wait(&bar.full[st], (g / kStages) & 1, &never);
+            }
+        }
+        if (abort_s) atomicOr(a.status, kStatusWaitExpired);
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (!abort_s) {
-        // Eq. 3-4: the block's windows (its first key is a multiple of omega)
-        const int w_begin = j_begin / s.omega;
-        const int n_win = (j_end - j_begin + s.omega - 1) / s.omega;
-        for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
-            const int lo = lw * s.omega;
-            const int size = min(s.omega, (j_end - j_begin) - lo);
-            a.window_scores[(size_t)unit * s.kw_max + w_begin + lw] = pool_top_p(t_chunk + lo, size, s.p);
-        }
-    } else if (threadIdx.x == 0) {
-        atomicOr(a.status, kStatusWaitExpired);
-    }
-    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -526,9 +674,16 @@ bool make_key_tensor_map(const KShape &ks, const void *k, CUtensorMap *tmap, int
     return true;
 }
 
-int device_cc_major()
+// what the launcher needs to know about the current device and its kernels, looked up once
+struct DeviceInfo {
+    int cc_major = -1;
+    int sm_count = 0;
+    int cooperative = 0;
+    int blocks_per_sm[2] = {-1, -1};   // resident blocks of each instantiation at its largest footprint
+};
+DeviceInfo &device_info()
 {
-    static int major = -1;
+    static DeviceInfo info;
     static std::once_flag once;
     std::call_once(once, [] {
         int dev = 0;
@@ -537,72 +692,97 @@ int device_cc_major()
             return;
         }
         int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess) major = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess) info.cc_major = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) info.sm_count = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess) info.cooperative = v;
     });
-    return major;
+    return info;
+}
+
+size_t tc_smem_bytes(int kblocks, int mb)
+{
+    return 1024 + (size_t)kblocks * mb * 128 * 128 + (size_t)kStages * kblocks * kRegion;
 }
 
 }  // namespace
 
 bool score_tc_supported(const KShape &ks, int dtype)
 {
+    const DeviceInfo &di = device_info();
     return dtype == WKV_BF16 && (ks.d == 64 || ks.d == 128) && ks.R <= 256 && ks.omega <= kTcMaxWindow &&
-           device_cc_major() == 10;
+           di.cc_major == 10 && di.cooperative && di.sm_count > 0;
 }
 
 int launch_score_tc(const KShape &ks, const void *q, const void *k, float *window_scores, float *token_scores,
-                    void *workspace, const Workspace &ws, cudaStream_t stream)
+                    int *window_idx, int *kept_len, void *workspace, const Workspace &ws, cudaStream_t stream)
 {
-    if (ks.max_seqlen - ks.alpha <= 0) return WKV_OK;
     alignas(64) CUtensorMap tmap;
     int slot[3] = {1, 2, 3};
     if (!make_key_tensor_map(ks, k, &tmap, slot)) return WKV_ERR_UNSUPPORTED;
+    DeviceInfo &di = device_info();
 
     TcArgs a;
     a.s = ks;
     a.stats = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + ws.stats_off);
     a.window_scores = window_scores;
     a.token_scores = token_scores;
+    a.window_idx = window_idx;
+    a.kept_len = kept_len;
     a.status = reinterpret_cast<int *>(static_cast<char *>(workspace) + ws.status_off);
+    a.sync = reinterpret_cast<int *>(static_cast<char *>(workspace) + ws.sync_off);
     a.n_stat_chunks = ws.n_stat_chunks;
     a.r_pad = ws.r_pad;
     const int units = ks.batch * ks.hkv;
-    a.chunks_per_unit = tc_chunks_per_unit(units, ks.max_seqlen);
+    const TcPlan plan = tc_plan(units, ks.max_seqlen, ks.d);
+    a.chunks_per_unit = plan.chunks_per_unit;
+    a.units_per_wave = plan.units_per_wave;
     a.kblocks = ks.d / 64;
     a.slot_tok = slot[0];
     a.slot_h = slot[1];
     a.slot_b = slot[2];
     a.r16 = (ks.R + 15) / 16 * 16;
-    int cols = 32;
-    while (cols < 2 * a.r16) cols <<= 1;
-    a.tmem_cols = cols;
 
     const int mb = ks.R > 128 ? 2 : 1;
-    const size_t stage_bytes = (size_t)kStages * a.kblocks * kRegion;
-    const size_t smem1 = 1024 + (size_t)a.kblocks * mb * 128 * 128 + stage_bytes;
-    const size_t smem2 = 2048 + (size_t)a.kblocks * a.r16 * 128 + stage_bytes;
-    dim3 grid(a.chunks_per_unit, units);
-    cudaError_t err;
-    const __nv_bfloat16 *qp = static_cast<const __nv_bfloat16 *>(q);
-    if (mb == 1) {
-        err = cudaFuncSetAttribute(score_stats_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
-        if (err == cudaSuccess) score_stats_tc<1><<<grid, kThreads, smem1, stream>>>(tmap, a, qp);
-    } else {
-        err = cudaFuncSetAttribute(score_stats_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
-        if (err == cudaSuccess) score_stats_tc<2><<<grid, kThreads, smem1, stream>>>(tmap, a, qp);
+    const int threads = block_threads(mb);
+    const size_t smem = tc_smem_bytes(a.kblocks, mb);
+    const void *fn = mb == 1 ? reinterpret_cast<const void *>(score_windows_tc<1>)
+                             : reinterpret_cast<const void *>(score_windows_tc<2>);
+    cudaError_t err = cudaSuccess;
+    if (di.blocks_per_sm[mb - 1] < 0) {
+        // once per instantiation: allow its largest shared-memory request (head_dim 128) and ask how
+        // many of its blocks an SM holds at that size
+        const size_t smem_max = tc_smem_bytes(2, mb);
+        err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        if (err == cudaSuccess)
+            err = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        int occ = 0;
+        if (err == cudaSuccess) err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, threads, smem_max);
+        if (err == cudaSuccess) {
+            if (occ < 1) {
+                cudaFuncAttributes fa;
+                (void)cudaFuncGetAttributes(&fa, fn);
+                set_error_detail("tensor-core score kernel does not fit an SM (%d threads, %d registers, %zu + %zu bytes "
+                                 "of shared memory)", threads, fa.numRegs, smem_max, fa.sharedSizeBytes);
+                return WKV_ERR_CUDA;
+            }
+            di.blocks_per_sm[mb - 1] = occ;
+        }
     }
-    if (err == cudaSuccess) err = cudaGetLastError();
-    if (err == cudaSuccess)
-        err = cudaFuncSetAttribute(score_pool_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    // persistent blocks, one per SM at most; every block of a cooperative launch is resident, which
+    // the grid barrier between the sweeps relies on
+    int grid = plan.units_per_wave * plan.chunks_per_unit;
+    if (grid > di.sm_count) grid = di.sm_count;
+    const __nv_bfloat16 *qp = static_cast<const __nv_bfloat16 *>(q);
     if (err == cudaSuccess) {
-        score_pool_tc<<<grid, kThreads, smem2, stream>>>(tmap, a, qp);
-        err = cudaGetLastError();
+        void *params[3] = {&tmap, &a, &qp};
+        err = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(threads), params, smem, stream);
     }
     if (err != cudaSuccess) {
-        set_error_detail("tensor-core score kernels: %s", cudaGetErrorString(err));
+        set_error_detail("tensor-core score kernel (grid %d x %d threads, %zu bytes of shared memory): %s", grid,
+                         threads, smem, cudaGetErrorString(err));
         return WKV_ERR_CUDA;
     }
-    count_launches(2);
+    count_launches(1);
     return WKV_OK;
 }
 

@@ -33,11 +33,13 @@ Workspace plan_workspace(const KShape &ks)
     const size_t units = (size_t)ks.batch * ks.hkv;
     w.r_pad = (ks.R + 63) / 64 * 64;
     w.n_stat_chunks = (ks.max_seqlen + kStatChunk - 1) / kStatChunk;
-    const int tc_chunks = tc_chunks_per_unit((int)units, ks.max_seqlen);
+    const int tc_chunks = tc_plan((int)units, ks.max_seqlen, ks.d).chunks_per_unit;
     if (tc_chunks > w.n_stat_chunks) w.n_stat_chunks = tc_chunks;
     size_t off = 0;
     w.status_off = off;
-    off = 256;
+    off = 64;
+    w.sync_off = off;
+    off = align_up(off + (16 + units) * sizeof(int), 256);
     w.stats_off = off;
     off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
     w.lse_off = off;
@@ -208,7 +210,8 @@ static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace
 }
 
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
-                    float *window_scores, float *token_scores, void *workspace, cudaStream_t stream)
+             float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
+             cudaStream_t stream)
 {
     if (!aligned16(q) || !aligned16(k)) {
         set_error_detail("q_obs / k_leader not 16-byte aligned");
@@ -218,13 +221,16 @@ int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const vo
     int st = pick_score_impl(s, ks, ws, use_tc);
     if (st != WKV_OK) return st;
     if (use_tc) {
-        st = launch_score_tc(ks, q, k, window_scores, token_scores, workspace, ws, stream);
+        st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream);
         // a key layout that no tensor map can describe is served by the CUDA-core kernels
         if (st != WKV_ERR_UNSUPPORTED || s->score_impl == WKV_SCORE_TCGEN05) return st;
         if (score_simt_smem_bytes(ks, ws.r_pad) > 227u * 1024u) return st;
     }
-    return check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream),
-                      "score kernels");
+    st = check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream),
+                    "score kernels");
+    if (st == WKV_OK && window_idx)
+        st = check_cuda(launch_topk(ks, window_scores, window_idx, kept_len, stream), "selection kernel");
+    return st;
 }
 
 static int fill_table(int n_layers, const void *const *k_layers, const void *const *v_layers,
@@ -323,7 +329,7 @@ int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leade
     const Workspace ws = plan_workspace(ks);
     st = check_workspace(ws, workspace, workspace_bytes);
     if (st != WKV_OK) return st;
-    return do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, workspace,
+    return do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, nullptr, nullptr, workspace,
                     static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -393,9 +399,7 @@ int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_l
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float *scores = window_scores ? window_scores
                                   : reinterpret_cast<float *>(static_cast<char *>(workspace) + ws.scores_off);
-    st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, workspace, stream);
-    if (st != WKV_OK) return st;
-    st = check_cuda(launch_topk(ks, scores, window_idx, kept_len, stream), "selection kernel");
+    st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, window_idx, kept_len, workspace, stream);
     if (st != WKV_OK) return st;
     return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
                                     keep_capacity, stream),

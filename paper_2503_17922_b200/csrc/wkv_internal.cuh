@@ -64,6 +64,7 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
     size_t status_off;   // int: device status word, only ever OR-ed by the kernels (0 = no error)
+    size_t sync_off;     // int [16 + units]: grid-barrier count and generation, per-unit tickets (self-resetting)
     size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
     size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
     size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none
@@ -81,15 +82,29 @@ constexpr int kTcMaxChunkTiles = 16;
 constexpr int kTcTargetBlocks = 148;
 constexpr int kTcMaxWindow = 1024;
 
-// blocks per unit (grid.x) of the tensor-core kernels
-__host__ __device__ inline int tc_chunks_per_unit(int units, int max_seqlen)
+// The tensor-core kernel works through the units in waves whose keys fit the L2 cache together, so
+// that the second sweep over a wave's keys is served from L2.  kTcWaveBytes is the budget.
+constexpr long long kTcWaveBytes = 80ll << 20;
+
+struct TcPlan {
+    int units_per_wave;   // units swept together
+    int chunks_per_unit;  // work items per unit
+};
+__host__ __device__ inline TcPlan tc_plan(int units, int max_seqlen, int head_dim)
 {
+    TcPlan p;
+    const long long unit_bytes = (long long)max_seqlen * head_dim * 2;
+    long long upw = kTcWaveBytes / (unit_bytes > 0 ? unit_bytes : 1);
+    if (upw < 1) upw = 1;
+    if (upw > units) upw = units;
+    p.units_per_wave = (int)upw;
     const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
-    int a = kTcTargetBlocks / units;
+    int a = kTcTargetBlocks / p.units_per_wave;
     const int b = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
     if (a < 1) a = 1;
     if (a > max_tiles) a = max_tiles;
-    return a > b ? a : b;
+    p.chunks_per_unit = a > b ? a : b;
+    return p;
 }
 // keys per block when `n_keys` keys are split over `chunks` blocks in whole tiles, rounded up to a
 // multiple of `align` (1 for the statistics sweep, omega for the scoring sweep)
@@ -111,8 +126,9 @@ cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const 
                               float *window_scores, float *token_scores,
                               void *workspace, const Workspace &ws, cudaStream_t stream);
 bool score_tc_supported(const KShape &ks, int dtype);
+// window_idx / kept_len non-null: the selection is fused into the same launch
 int launch_score_tc(const KShape &ks, const void *q, const void *k,
-                    float *window_scores, float *token_scores,
+                    float *window_scores, float *token_scores, int *window_idx, int *kept_len,
                     void *workspace, const Workspace &ws, cudaStream_t stream);
 cudaError_t launch_topk(const KShape &ks, const float *window_scores, int *window_idx, int *kept_len,
                         cudaStream_t stream);
@@ -157,8 +173,10 @@ __device__ inline float pool_top_p(const float *w, int size, int p)
 // host side of the boundary, shared by the translation units that export entry points
 int resolve(const wkv_shape *s, KShape &ks);            // validates the shape, fills the kernel-side copy
 int check_cuda(cudaError_t e, const char *what);         // cudaError_t -> wkv_status with detail
+// scoring; with window_idx / kept_len non-null also the selection (one launch on the tensor-core path)
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
-             float *window_scores, float *token_scores, void *workspace, cudaStream_t stream);
+             float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
+             cudaStream_t stream);
 
 void count_launches(int n);
 void set_error_detail(const char *fmt, ...);

@@ -254,7 +254,7 @@ def test_launches_are_counted_and_errors_raise():
     w = small()
     before = binding.wkv_launch_count()
     pu.run_gpu_group(w, wl.make_group(w, 0))
-    assert binding.wkv_launch_count() - before >= 3
+    assert binding.wkv_launch_count() - before >= 2     # fused score+selection launch, gather launch
     prob = binding.Problem.from_workload(w)
     with pytest.raises(binding.WkvError):
         binding.wkv_score_windows(prob, None, None, None, None, prob.alloc_workspace())
