@@ -32,6 +32,7 @@
 
 #include <algorithm>
 #include <mutex>
+#include <type_traits>
 
 namespace wkv {
 namespace {
@@ -45,7 +46,7 @@ __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
 constexpr int kChunkCap = kTcMaxChunkTiles * kTile + kTcMaxWindow;   // token scores a block may hold
-constexpr int kSyncTickets = 16;                         // sync[0] barrier count, sync[1] generation, then tickets
+constexpr int kSyncTickets = 16;                         // sync[0] grid-barrier word, tickets from sync[16]
 
 struct TcArgs {
     KShape s;
@@ -104,9 +105,10 @@ __device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
     if (lane == 0) mbar_arrive(bar);
 }
 
-// Grid-wide barrier of a cooperative launch (all blocks resident).  sync[0] counts arrivals and is
-// reset by the last arriver, sync[1] is the generation the others wait on.  Bounded: a block that
-// waits longer than two seconds gives up, sets its abort flag and the caller tears the block down.
+// Grid-wide barrier of a cooperative launch (all blocks resident).  One word: arrivals in the low 16
+// bits, generation above; the last arriver clears the count and bumps the generation in one atomic.
+// Bounded: a block that waits longer than two seconds gives up, sets its abort flag and the caller
+// tears the block down.
 __device__ __forceinline__ int ld_acquire_gpu(const int *p)
 {
     int v;
@@ -115,21 +117,26 @@ __device__ __forceinline__ int ld_acquire_gpu(const int *p)
 }
 __device__ __forceinline__ void grid_barrier(int *sync, int n_blocks, volatile int *abort_flag)
 {
-    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0 && !*abort_flag) {
-        const int gen = ld_acquire_gpu(&sync[1]);
-        if (atomicAdd(&sync[0], 1) == n_blocks - 1) {
-            atomicExch(&sync[0], 0);
+        // the fence of thread 0 is cumulative: it also publishes what the other threads of the block
+        // wrote before the block barrier above
+        __threadfence();
+        const int old = atomicAdd(sync, 1);
+        if ((old & 0xffff) == n_blocks - 1) {
             __threadfence();
-            atomicAdd(&sync[1], 1);
+            atomicAdd(sync, 0x10000 - n_blocks);
         } else {
-            const unsigned long long t0 = global_timer_ns();
-            while (ld_acquire_gpu(&sync[1]) == gen) {
-                __nanosleep(64);
-                if (global_timer_ns() - t0 > 2 * kWaitLimitNs) {
-                    *abort_flag = 1;
-                    break;
+            const int gen = old >> 16;
+            unsigned long long t0 = 0;
+            for (uint32_t spin = 1; (ld_acquire_gpu(sync) >> 16) == gen; ++spin) {
+                if ((spin & 1023u) == 0u) {
+                    const unsigned long long now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > 2 * kWaitLimitNs) {
+                        *abort_flag = 1;
+                        break;
+                    }
                 }
             }
         }
@@ -195,31 +202,26 @@ __device__ __forceinline__ void score_accumulate(const float (&v)[N], const floa
     }
 }
 
-// Eq. 4 for windows whose length omega is a power of two <= 32: a warp takes 32/omega windows at a
-// time, one lane per token.  The rank of a token inside its window (value descending, position
-// ascending) comes from omega shuffles; the p best are summed by a butterfly in a fixed order.
-__device__ __forceinline__ void pool_windows_warp(const float *t_chunk, int n_tok, int omega, int p, float *out,
-                                                  int warp, int n_warps, int lane)
+// Eq. 4 for one window of compile-time length by one thread: the values sit in registers, the rank
+// of each (value descending, position ascending) comes from omega*omega independent comparisons, and
+// the p best are summed in position order.
+template <int omega>
+__device__ __forceinline__ float pool_window_regs(const float *w, int size, int p)
 {
-    const int per_warp = 32 / omega;
-    const int n_win = (n_tok + omega - 1) / omega;
-    const int e = lane % omega, sub = lane / omega;
-    for (int w0 = warp * per_warp; w0 < n_win; w0 += n_warps * per_warp) {
-        const int w = w0 + sub;
-        const int j = w * omega + e;
-        const bool valid = w < n_win && j < n_tok;
-        const float v = valid ? t_chunk[j] : -INFINITY;
+    float v[omega];
+#pragma unroll
+    for (int x = 0; x < omega; ++x) v[x] = x < size ? w[x] : -INFINITY;
+    const int p_eff = p < size ? p : size;
+    float acc = 0.f;
+#pragma unroll
+    for (int x = 0; x < omega; ++x) {
         int rank = 0;
-        for (int x = 0; x < omega; ++x) {
-            const float o = __shfl_sync(0xffffffffu, v, sub * omega + x);
-            rank += (o > v || (o == v && x < e)) ? 1 : 0;
-        }
-        const int size = w < n_win ? min(omega, n_tok - w * omega) : 1;
-        const int p_eff = p < size ? p : size;
-        float acc = (valid && rank < p_eff) ? v : 0.f;
-        for (int o = 1; o < omega; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (e == 0 && w < n_win) out[w] = acc / (float)p_eff;
+#pragma unroll
+        for (int y = 0; y < omega; ++y)
+            if (y != x) rank += (int)(v[y] > v[x]) | ((int)(v[y] == v[x]) & (int)(y < x));
+        acc += (x < size && rank < p_eff) ? v[x] : 0.f;
     }
+    return acc / (float)p_eff;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -284,10 +286,15 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.chunk = chunk;
         im.b = unit / s.hkv;
         im.h = unit % s.hkv;
-        const SeqInfo si = seq_info(s, im.b);
-        im.n = si.n;
-        im.n_r = si.n - s.alpha;
-        im.off = si.off;
+        if (s.cu) {
+            const int lo = s.cu[im.b];
+            im.n = s.cu[im.b + 1] - lo;
+            im.off = lo;
+        } else {
+            im.n = s.max_seqlen;
+            im.off = 0;
+        }
+        im.n_r = im.n - s.alpha;
         const int n_keys = review_only ? im.n_r : im.n;
         const int len = tc_chunk_len(n_keys > 0 ? n_keys : 1, cpu, review_only ? s.omega : 1);
         im.j_begin = chunk * len;
@@ -295,22 +302,40 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.n_tiles = im.j_end > im.j_begin ? (im.j_end - im.j_begin + kTile - 1) / kTile : 0;
     };
 
+    // Called by every warp except the producer (which has no use for Q and starts streaming keys at
+    // once); ends with a barrier among those warps.  Four loads are in flight per thread.
+    constexpr int kLoaders = kThreads - 32;
     auto load_q_image = [&](const Item &im) {
-        if (q_unit_loaded == im.unit) return;
-        q_unit_loaded = im.unit;
-        const __nv_bfloat16 *q_unit = q + im.b * s.qsb + (long long)im.h * s.G * s.qsh;
-        const int vec_per_row = s.d / 8;
-        for (int idx = threadIdx.x; idx < q_rows * vec_per_row; idx += kThreads) {
-            const int r = idx / vec_per_row, cc = idx % vec_per_row;
-            const int rq = r % Rp;
-            int4 v = make_int4(0, 0, 0, 0);
-            if (rq < s.R) {
-                const int g = rq / s.alpha, i = rq % s.alpha;
-                v = *reinterpret_cast<const int4 *>(q_unit + g * s.qsh + i * s.qst + cc * 8);
+        if (q_unit_loaded != im.unit) {
+            const __nv_bfloat16 *q_unit = q + im.b * s.qsb + (long long)im.h * s.G * s.qsh;
+            const int vshift = s.d == 128 ? 4 : 3;            // log2(16-byte vectors per row)
+            const int total = q_rows << vshift;
+            for (int base = threadIdx.x - 32; base < total; base += kLoaders * 4) {
+                int4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int idx = base + u * kLoaders;
+                    v[u] = make_int4(0, 0, 0, 0);
+                    if (idx < total) {
+                        const int rq = (idx >> vshift) % Rp, cc = idx & ((1 << vshift) - 1);
+                        if (rq < s.R) {
+                            const int g = rq / s.alpha, i = rq - g * s.alpha;
+                            v[u] = __ldg(reinterpret_cast<const int4 *>(q_unit + g * s.qsh + i * s.qst + cc * 8));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int idx = base + u * kLoaders;
+                    if (idx < total) {
+                        const int r = idx >> vshift, cc = idx & ((1 << vshift) - 1);
+                        *reinterpret_cast<int4 *>(q_img + (cc >> 3) * q_region + swz128_offset(r, cc & 7)) = v[u];
+                    }
+                }
             }
-            *reinterpret_cast<int4 *>(q_img + (cc >> 3) * q_region + swz128_offset(r, cc & 7)) = v;
+            fence_proxy_async_smem();
         }
-        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
     };
 
     // producer: the item's key tiles into the stage ring (the block-wide tile counter `it` keeps the phases)
@@ -332,33 +357,45 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         }
     };
 
-    // MMA issue for one item.  sweep 1: D[rows, keys] = Q K^T (MB row blocks); sweep 2: D[keys, rows] = K Q^T
+    // MMA issue for one item.  sweep 1: D[rows, keys] = Q K^T (MB row blocks); sweep 2: D[keys, rows] = K Q^T.
+    // One thread issues everything, so its instruction count per tile is on the critical path: the
+    // matrix descriptors of Q and of stage 0 are built once, and every k-step only adds a
+    // compile-time constant to the address field (the fields above it never change).
+    const uint64_t q_desc0 = umma_desc_sw128(smem_u32(q_img));
+    const uint64_t k_desc0 = umma_desc_sw128(smem_u32(k_stage0));
+    auto issue_tile = [&](auto ksteps_tag, uint32_t d_tmem, uint64_t k_desc, uint32_t idesc, bool sweep2) {
+        constexpr int KSTEPS = decltype(ksteps_tag)::value;
+        if (sweep2) {
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                const uint32_t qo = (uint32_t)((ks >> 2) * q_region + (ks & 3) * 32) >> 4;
+                const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
+                umma_bf16(d_tmem, k_desc + ko, q_desc0 + qo, idesc, ks > 0);
+            }
+        } else {
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    const uint32_t qo = (uint32_t)((ks >> 2) * q_region + mb * kRegion + (ks & 3) * 32) >> 4;
+                    const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
+                    umma_bf16(d_tmem + mb * 128, q_desc0 + qo, k_desc + ko, idesc, ks > 0);
+                }
+        }
+    };
     auto issue_mma = [&](const Item &im, bool sweep2) {
-        const uint32_t q_addr = smem_u32(q_img);
         const uint32_t idesc = sweep2 ? umma_idesc_bf16(128, a.r16) : umma_idesc_bf16(128, kTile);
+        const uint32_t stage_step = (uint32_t)stage_bytes >> 4;
         for (int t = 0; t < im.n_tiles; ++t) {
             const uint32_t g = it + t;
             const int st = g % kStages, buf = g % NG;
             if (!mbar_wait(&bar.full[st], (g / kStages) & 1, &abort_s)) return;
             if (g >= NG && !mbar_wait(&bar.tempty[buf], ((g / NG) - 1) & 1, &abort_s)) return;
             tc_fence_after_sync();
-            const uint32_t k_addr = smem_u32(k_stage0 + st * stage_bytes);
+            const uint64_t k_desc = k_desc0 + (uint64_t)(st * stage_step);
             const uint32_t d_tmem = tmem_base + buf * buf_cols;
-            if (sweep2) {
-                for (int ks = 0; ks < ksteps; ++ks) {
-                    const uint32_t kb = ks >> 2, sub = (ks & 3) * 32;
-                    umma_bf16(d_tmem, umma_desc_sw128(k_addr + kb * kRegion + sub),
-                              umma_desc_sw128(q_addr + kb * q_region + sub), idesc, ks > 0);
-                }
-            } else {
-#pragma unroll
-                for (int mb = 0; mb < MB; ++mb)
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint32_t kb = ks >> 2, sub = (ks & 3) * 32;
-                        umma_bf16(d_tmem + mb * 128, umma_desc_sw128(q_addr + kb * q_region + mb * kRegion + sub),
-                                  umma_desc_sw128(k_addr + kb * kRegion + sub), idesc, ks > 0);
-                    }
-            }
+            if (ksteps == 8) issue_tile(std::integral_constant<int, 8>{}, d_tmem, k_desc, idesc, sweep2);
+            else issue_tile(std::integral_constant<int, 4>{}, d_tmem, k_desc, idesc, sweep2);
             umma_commit(&bar.empty[st]);
             umma_commit(&bar.tfull[buf]);
         }
@@ -450,15 +487,17 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 for (int r = threadIdx.x; r < a.r_pad; r += kThreads) out[r] = make_float2(-INFINITY, 0.f);
                 continue;
             }
-            load_q_image(im);
-            __syncthreads();
             if (warp == 0) {
                 if (lane == 0) produce(im);
-            } else if (warp == 1) {
-                if (lane == 0) issue_mma(im, false);
             } else {
-                compute_stats(im);
+                load_q_image(im);
+                if (warp == 1) {
+                    if (lane == 0) issue_mma(im, false);
+                } else {
+                    compute_stats(im);
+                }
             }
+            q_unit_loaded = im.unit;
             it += im.n_tiles;
             tc_fence_before_sync();
             __syncthreads();
@@ -477,12 +516,13 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                     for (int g = 0; g < NG; ++g)
                         for (int cp = 0; cp < copies; ++cp) {
                             const float2 p = part[g][mb][base + cp * Rp];
-                            if (p.y > 0.f) sum += p.y * exp2f((p.x - M) * c);
+                            if (p.y > 0.f) sum += p.y * fast_exp2((p.x - M) * c);
                         }
                     res = make_float2(M * c, sum);
                 }
                 out[r] = res;
             }
+            __syncthreads();   // `part` is rewritten by the next item
         }
 
         grid_barrier(a.sync, gridDim.x, &abort_s);
@@ -503,38 +543,70 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 }
                 continue;
             }
-            load_q_image(im);
-            {
-                // Eq. 1's normaliser of every row: merge the partial statistics of the unit's chunks
-                const int len1 = tc_chunk_len(im.n, cpu, 1);
-                const int used = (im.n + len1 - 1) / len1;
-                for (int r = threadIdx.x; r < 256; r += kThreads) {
-                    float v = -INFINITY;
+            if (warp == 0) {
+                if (lane == 0) produce(im);
+            } else {
+                load_q_image(im);
+                // Eq. 1's normaliser of every row: merge the partial statistics of the unit's chunks.
+                // kMergers threads share a row (each takes every kMergers-th chunk), then one of them
+                // merges their results; both steps in a fixed order.
+                constexpr int kMergers = kLoaders / q_rows;
+                float2 *merged = &part[0][0][0];
+                const int tl = threadIdx.x - 32;
+                if (tl < kMergers * q_rows) {
+                    const int r = tl % q_rows, mp = tl / q_rows;
+                    float M = -INFINITY, sum = 0.f;
                     if (r < s.R) {
+                        const int len1 = tc_chunk_len(im.n, cpu, 1);
+                        const int used = (im.n + len1 - 1) / len1;
                         const float2 *st = a.stats + (size_t)im.unit * a.n_stat_chunks * a.r_pad + r;
+                        for (int c0 = mp; c0 < used; c0 += 8 * kMergers) {
+                            float2 p[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int cidx = c0 + u * kMergers;
+                                p[u] = cidx < used ? __ldcg(st + (size_t)cidx * a.r_pad) : make_float2(-INFINITY, 0.f);
+                            }
+                            float Mn = M;
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, p[u].x);
+                            if (Mn > -INFINITY) {
+                                sum *= fast_exp2(M - Mn);
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    if (p[u].y > 0.f) sum += p[u].y * fast_exp2(p[u].x - Mn);
+                                M = Mn;
+                            }
+                        }
+                    }
+                    merged[mp * q_rows + r] = make_float2(M, sum);
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
+                if (tl < 256) {
+                    float v = -INFINITY;
+                    if (tl < s.R) {
                         float M = -INFINITY, sum = 0.f;
-#pragma unroll 6
-                        for (int cidx = 0; cidx < used; ++cidx) {
-                            const float2 p = __ldcg(st + (size_t)cidx * a.r_pad);
+#pragma unroll
+                        for (int mp = 0; mp < kMergers; ++mp) {
+                            const float2 p = merged[mp * q_rows + tl];
                             if (p.y > 0.f) {
                                 const float Mn = fmaxf(M, p.x);
-                                sum = sum * exp2f(M - Mn) + p.y * exp2f(p.x - Mn);
+                                sum = sum * fast_exp2(M - Mn) + p.y * fast_exp2(p.x - Mn);
                                 M = Mn;
                             }
                         }
                         if (sum > 0.f) v = -(M + log2f(sum));
                     }
-                    neg_lse2[r] = v;
+                    neg_lse2[tl] = v;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
+                if (warp == 1) {
+                    if (lane == 0) issue_mma(im, true);
+                } else {
+                    compute_scores(im);
                 }
             }
-            __syncthreads();
-            if (warp == 0) {
-                if (lane == 0) produce(im);
-            } else if (warp == 1) {
-                if (lane == 0) issue_mma(im, true);
-            } else {
-                compute_scores(im);
-            }
+            q_unit_loaded = im.unit;
             it += im.n_tiles;
             tc_fence_before_sync();
             __syncthreads();
@@ -544,10 +616,19 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             {
                 const int n_tok = im.j_end - im.j_begin;
                 float *ws_out = a.window_scores + (size_t)im.unit * s.kw_max + im.j_begin / s.omega;
-                if (s.omega <= 32 && (s.omega & (s.omega - 1)) == 0) {
-                    pool_windows_warp(t_chunk, n_tok, s.omega, s.p, ws_out, warp, kThreads / 32, lane);
-                } else {
-                    const int n_win = (n_tok + s.omega - 1) / s.omega;
+                const int n_win = (n_tok + s.omega - 1) / s.omega;
+                if (s.omega == 16 || s.omega == 8 || s.omega == 32 || s.omega == 4) {
+                    for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
+                        const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
+                        float r;
+                        if (s.omega == 16) r = pool_window_regs<16>(t_chunk + lo, size, s.p);
+                        else if (s.omega == 8) r = pool_window_regs<8>(t_chunk + lo, size, s.p);
+                        else if (s.omega == 32) r = pool_window_regs<32>(t_chunk + lo, size, s.p);
+                        else r = pool_window_regs<4>(t_chunk + lo, size, s.p);
+                        ws_out[lw] = r;
+                    }
+                }
+                else {
                     for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
                         const int lo = lw * s.omega;
                         ws_out[lw] = pool_top_p(t_chunk + lo, min(s.omega, n_tok - lo), s.p);
@@ -558,13 +639,15 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 // the block that completes the unit's last windows selects for the unit
                 const int len2 = tc_chunk_len(im.n_r, cpu, s.omega);
                 const int used2 = (im.n_r + len2 - 1) / len2;
-                __threadfence();
                 __syncthreads();
                 if (threadIdx.x == 0) {
+                    __threadfence();   // cumulative: publishes the window scores the whole block wrote
                     int *ticket = a.sync + kSyncTickets + im.unit;
                     const int last = atomicAdd(ticket, 1) == used2 - 1;
-                    if (last) atomicExch(ticket, 0);
-                    __threadfence();
+                    if (last) {
+                        atomicExch(ticket, 0);
+                        __threadfence();
+                    }
                     flag_s = last;
                 }
                 __syncthreads();

@@ -55,32 +55,55 @@ __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total
 // All NT threads of the block call this.  `sc` are the unit's kw window scores (read through L2,
 // so scores written by other blocks of the same grid are seen once the caller has synchronised
 // with them), `out` receives k ascending indices followed by -1 up to k_max.
-template <int NT>
-__device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, int k_max, int *out,
-                                  int *kept_len_out, int n, int alpha, int omega)
+// Thread t owns the windows [t*E, (t+1)*E), E = ceil(kw / NT).  With E <= kTopkRegs the keys are
+// read once and stay in registers through the four radix passes and the compaction (one trip to
+// L2 instead of six); longer lists are re-read.
+constexpr int kTopkRegs = 8;
+
+template <int NT, bool IN_REGS>
+__device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, int kw, int k, int *out,
+                                                 int *kept_len_out, int n, int alpha, int omega, int obs_rows)
 {
-    static_assert(NT % 32 == 0 && NT <= 1024, "block size");
-    for (int x = (k > 0 ? k : 0) + threadIdx.x; x < k_max; x += NT) out[x] = -1;
-    const int obs_rows = n < alpha ? n : alpha;
-    if (k <= 0) {
-        if (threadIdx.x == 0) *kept_len_out = obs_rows;
-        return;
+    const int E = (kw + NT - 1) / NT;
+    const int w_lo = min(kw, (int)threadIdx.x * E), w_hi = min(kw, w_lo + E);
+    unsigned keys[kTopkRegs];
+    if (IN_REGS) {
+#pragma unroll
+        for (int e = 0; e < kTopkRegs; ++e) keys[e] = w_lo + e < w_hi ? topk_order_key(__ldcg(sc + w_lo + e)) : 0u;
     }
+    auto key_at = [&](int e) -> unsigned { return IN_REGS ? keys[e] : topk_order_key(__ldcg(sc + w_lo + e)); };
+
     // ---- radix select: key of the k-th largest score --------------------------------
     if (threadIdx.x == 0) {
         sm.prefix = 0u;
         sm.remaining = k;
         sm.last_selected = 0;
     }
+    for (int x = threadIdx.x; x < 256; x += NT) sm.hist[x] = 0;
+    __syncthreads();
     unsigned mask = 0u;
     for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int x = threadIdx.x; x < 256; x += NT) sm.hist[x] = 0;
-        __syncthreads();
         const unsigned prefix = sm.prefix;
         const int remaining = sm.remaining;
-        for (int w = threadIdx.x; w < kw; w += NT) {
-            const unsigned key = topk_order_key(__ldcg(sc + w));
-            if ((key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 0xffu], 1);
+        // window scores share sign and exponent, so most keys of a pass fall into very few bins:
+        // the lanes of a warp that hit the same bin are counted by one of them
+#pragma unroll
+        for (int e = 0; e < (IN_REGS ? kTopkRegs : E); ++e) {
+            if (IN_REGS && e >= E) break;   // uniform: E is the same for every thread
+            unsigned bin = 256u;            // not taking part in this pass
+            if (w_lo + e < w_hi) {
+                const unsigned key = key_at(e);
+                if ((key & mask) == prefix) bin = (key >> shift) & 0xffu;
+            }
+            // the lanes that share the bin of the first participating lane are counted by that lane
+            const unsigned part = __ballot_sync(0xffffffffu, bin < 256u);
+            if (part) {
+                const int leader = __ffs(part) - 1;
+                const unsigned pivot = __shfl_sync(0xffffffffu, bin, leader);
+                const unsigned same = __ballot_sync(0xffffffffu, bin == pivot);
+                if ((int)(threadIdx.x & 31) == leader) atomicAdd(&sm.hist[pivot], __popc(same));
+                else if (bin < 256u && bin != pivot) atomicAdd(&sm.hist[bin], 1);
+            }
         }
         __syncthreads();
         if (threadIdx.x < 32) {
@@ -90,6 +113,7 @@ __device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, 
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 c[i] = sm.hist[lane * 8 + i];
+                sm.hist[lane * 8 + i] = 0;   // ready for the next pass (and the next call)
                 tot += c[i];
             }
             int incl = tot;   // inclusive suffix sum over the lanes (lane 31 holds the top bins)
@@ -120,23 +144,52 @@ __device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, 
     const int need_eq = sm.remaining;
 
     // ---- ordered compaction ----------------------------------------------------------
-    int eq_base = 0, out_base = 0;
-    for (int w0 = 0; w0 < kw; w0 += NT) {
-        const int w = w0 + threadIdx.x;
-        unsigned key = 0u;
-        const bool in = w < kw;
-        if (in) key = topk_order_key(__ldcg(sc + w));
-        const int is_eq = in && key == thr;
-        int eq_total, sel_total;
-        const int eq_rank = eq_base + topk_block_scan<NT>(is_eq, sm.warp_sums, eq_total);
-        const int sel = in && (key > thr || (is_eq && eq_rank < need_eq));
-        const int pos = out_base + topk_block_scan<NT>(sel, sm.warp_sums, sel_total);
-        if (sel) {
-            out[pos] = w;
-            if (w == kw - 1) sm.last_selected = 1;
+    int n_eq = 0, n_gt = 0;
+    if (IN_REGS) {
+#pragma unroll
+        for (int e = 0; e < kTopkRegs; ++e)
+            if (w_lo + e < w_hi) {
+                n_eq += keys[e] == thr;
+                n_gt += keys[e] > thr;
+            }
+    } else {
+        for (int e = 0; w_lo + e < w_hi; ++e) {
+            const unsigned key = key_at(e);
+            n_eq += key == thr;
+            n_gt += key > thr;
         }
-        eq_base += eq_total;
-        out_base += sel_total;
+    }
+    int eq_rank, pos;   // threshold keys before this thread; output position of its first selected window
+    if (IN_REGS) {
+        // at most NT * kTopkRegs < 2^15 windows: both counts travel through one scan
+        int total;
+        const int both = topk_block_scan<NT>((n_eq << 16) | n_gt, sm.warp_sums, total);
+        eq_rank = both >> 16;
+        pos = (both & 0xffff) + (eq_rank < need_eq ? eq_rank : need_eq);
+    } else {
+        int eq_total, sel_total;
+        eq_rank = topk_block_scan<NT>(n_eq, sm.warp_sums, eq_total);
+        int n_eq_taken = need_eq - eq_rank;
+        n_eq_taken = n_eq_taken < 0 ? 0 : (n_eq_taken > n_eq ? n_eq : n_eq_taken);
+        pos = topk_block_scan<NT>(n_gt + n_eq_taken, sm.warp_sums, sel_total);
+    }
+    auto emit = [&](int e, unsigned key) {
+        bool sel = key > thr;
+        if (key == thr) {
+            sel = eq_rank < need_eq;
+            ++eq_rank;
+        }
+        if (sel) {
+            out[pos++] = w_lo + e;
+            if (w_lo + e == kw - 1) sm.last_selected = 1;
+        }
+    };
+    if (IN_REGS) {
+#pragma unroll
+        for (int e = 0; e < kTopkRegs; ++e)
+            if (w_lo + e < w_hi) emit(e, keys[e]);
+    } else {
+        for (int e = 0; w_lo + e < w_hi; ++e) emit(e, key_at(e));
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -144,6 +197,23 @@ __device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, 
         const int last_size = n_r - (kw - 1) * omega;     // real size of the last window
         *kept_len_out = k * omega - (sm.last_selected ? omega - last_size : 0) + obs_rows;
     }
+}
+
+template <int NT>
+__device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, int k_max, int *out,
+                                  int *kept_len_out, int n, int alpha, int omega)
+{
+    static_assert(NT % 32 == 0 && NT <= 1024, "block size");
+    for (int x = (k > 0 ? k : 0) + threadIdx.x; x < k_max; x += NT) out[x] = -1;
+    const int obs_rows = n < alpha ? n : alpha;
+    if (k <= 0) {
+        if (threadIdx.x == 0) *kept_len_out = obs_rows;
+        return;
+    }
+    if ((kw + NT - 1) / NT <= kTopkRegs)
+        select_topk_impl<NT, true>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+    else
+        select_topk_impl<NT, false>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
 }
 
 }  // namespace wkv
