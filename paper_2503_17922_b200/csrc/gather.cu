@@ -1,16 +1,19 @@
-// Shared-index gather (section 2.2.2): copies, for every layer tensor of the group,
-// the rows of the selected review windows followed by the observation rows into
-// the compact cache.  Pure bit copy with 16-byte vector accesses; a row of d
-// elements is d*elem_bytes/16 vectors, consecutive threads take consecutive
-// vectors so both the reads (omega consecutive rows per window) and the writes
-// (consecutive output rows) are fully coalesced.
+// Shared-index gather (section 2.2.2): copies, for every layer tensor of the group, the rows of
+// the selected review windows followed by the observation rows into the compact cache.  Pure bit
+// copy with 16-byte vector accesses.
+//
+// The unit of work is one window (omega consecutive source rows = omega consecutive output rows)
+// of one unit of one tensor, taken by one warp: all its loads are issued before the first store
+// (up to 8 x 16 bytes in flight per lane), and the index arithmetic is done once per window, not
+// once per vector.  The observation rows are handled as extra windows behind the selected ones.
 #include "wkv_internal.cuh"
 
 namespace wkv {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;            // independent 16-byte loads in flight per thread
+constexpr int kWarps = kThreads / 32;
+constexpr int kBatch = 8;             // independent 16-byte loads in flight per lane
 
 struct GatherParams {
     KShape s;
@@ -19,11 +22,13 @@ struct GatherParams {
     const int *cu_out;
     int keep_capacity;
     int vec_per_row;                  // 16-byte vectors per row
+    int vec_shift;                    // log2(vec_per_row) when it is a power of two, else -1
     int elem_bytes;
-    int rows_per_block;               // output rows handled by one block
+    int slots_per_block;              // windows (selected + observation) handled by one block
+    int obs_slots;                    // ceil(alpha / omega)
 };
 
-__device__ inline int4 ld_stream(const int4 *p)
+__device__ __forceinline__ int4 ld_stream(const int4 *p)
 {
     int4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
@@ -31,18 +36,19 @@ __device__ inline int4 ld_stream(const int4 *p)
                  : "l"(p));
     return v;
 }
-__device__ inline void st_stream(int4 *p, const int4 &v)
+__device__ __forceinline__ void st_stream(int4 *p, const int4 &v)
 {
     asm volatile("st.global.L1::no_allocate.v4.s32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y),
                  "r"(v.z), "r"(v.w)
                  : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 gather_kv_kernel(const __grid_constant__ GatherParams prm)
 {
     const KShape &s = prm.s;
     const int unit = blockIdx.y, tensor = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = unit / s.hkv, h = unit % s.hkv;
     const SeqInfo si = seq_info(s, b);
     const int n = si.n;
@@ -51,15 +57,11 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
     const int k = num_selected(n, s.alpha, s.omega, si.budget);
     const int *idx = prm.window_idx + (size_t)unit * s.k_max;
 
-    // rows of the unit: the selected windows (only the last window of the sequence can be
-    // short, and it can only be the last selected one), then the observation rows
+    // rows of the unit: the selected windows (only the last window of the sequence can be short,
+    // and it can only be the last selected one), then the observation rows
     int review_rows = k * s.omega;
     if (k > 0 && idx[k - 1] == kw - 1) review_rows -= kw * s.omega - n_r;
-    const int total_rows = review_rows + (n - n_r);
-
-    const int row_begin = blockIdx.x * prm.rows_per_block;
-    if (row_begin >= total_rows) return;
-    const int row_end = min(total_rows, row_begin + prm.rows_per_block);
+    const int obs_rows = n - n_r;
 
     const int vpr = prm.vec_per_row;
     // strides are multiples of 16 bytes (checked on the host), so vector indexing is exact
@@ -77,31 +79,46 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
         dst = reinterpret_cast<int4 *>(prm.tab.dst[tensor]) + (long long)unit * prm.keep_capacity * vpr;
         dst_row_vecs = vpr;
     }
+    const bool src_dense = src_row_vecs == vpr, dst_dense = dst_row_vecs == vpr;
 
-    const int n_vec = (row_end - row_begin) * vpr;
-    for (int v0 = threadIdx.x; v0 < n_vec; v0 += kThreads * kUnroll) {
-        int4 val[kUnroll];
-        long long doff[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int v = v0 + u * kThreads;
-            if (v < n_vec) {
-                const int r = row_begin + v / vpr, c = v % vpr;
-                int src_row;
-                if (r < review_rows) {
-                    const int w = r / s.omega;
-                    src_row = idx[w] * s.omega + (r - w * s.omega);
-                } else {
-                    src_row = n_r + (r - review_rows);
-                }
-                val[u] = ld_stream(src + src_row * src_row_vecs + c);
-                doff[u] = r * dst_row_vecs + c;
-            }
+    const int slot_end = min(k + prm.obs_slots, (int)(blockIdx.x + 1) * prm.slots_per_block);
+    for (int slot = blockIdx.x * prm.slots_per_block + warp; slot < slot_end; slot += kWarps) {
+        int src_row0, dst_row0, n_rows;
+        if (slot < k) {
+            src_row0 = idx[slot] * s.omega;
+            n_rows = min(s.omega, n_r - src_row0);
+            dst_row0 = slot * s.omega;
+        } else {
+            const int o = (slot - k) * s.omega;
+            src_row0 = n_r + o;
+            n_rows = min(s.omega, obs_rows - o);
+            dst_row0 = review_rows + o;
         }
+        if (n_rows <= 0) continue;
+        const int4 *sp = src + src_row0 * src_row_vecs;
+        int4 *dp = dst + dst_row0 * dst_row_vecs;
+        const int n_vec = n_rows * vpr;
+        for (int v0 = lane; v0 < n_vec; v0 += 32 * kBatch) {
+            int4 val[kBatch];
+            int soff[kBatch], doff[kBatch];   // offsets inside one window: small
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int v = v0 + u * kThreads;
-            if (v < n_vec) st_stream(dst + doff[u], val[u]);
+            for (int u = 0; u < kBatch; ++u) {
+                const int v = v0 + u * 32;
+                if (v < n_vec) {
+                    soff[u] = v;
+                    doff[u] = v;
+                    if (!src_dense || !dst_dense) {
+                        const int r = prm.vec_shift >= 0 ? v >> prm.vec_shift : v / vpr;
+                        const int c = v - r * vpr;
+                        if (!src_dense) soff[u] = r * (int)src_row_vecs + c;
+                        if (!dst_dense) doff[u] = r * (int)dst_row_vecs + c;
+                    }
+                    val[u] = ld_stream(sp + soff[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                if (v0 + u * 32 < n_vec) st_stream(dp + doff[u], val[u]);
         }
     }
 }
@@ -119,14 +136,18 @@ cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const
     prm.cu_out = cu_out;
     prm.keep_capacity = keep_capacity;
     prm.vec_per_row = ks.d * elem_bytes / 16;
+    prm.vec_shift = -1;
+    for (int sh = 0; sh < 16; ++sh)
+        if ((1 << sh) == prm.vec_per_row) prm.vec_shift = sh;
     prm.elem_bytes = elem_bytes;
-    // each block moves about 64 KB so that a full-size group yields several waves of blocks
-    int rows = (64 * 1024) / (prm.vec_per_row * 16);
-    if (rows < 1) rows = 1;
-    prm.rows_per_block = rows;
-    // upper bound of rows per unit: all selected windows full + observation rows
-    const int max_rows = ks.k_max * ks.omega + ks.alpha;
-    dim3 grid((max_rows + rows - 1) / rows, ks.batch * ks.hkv, n_tensors);
+    prm.obs_slots = (ks.alpha + ks.omega - 1) / ks.omega;
+    // each warp moves a few windows; a block takes about 64 KB
+    const long long window_bytes = (long long)ks.omega * prm.vec_per_row * 16;
+    long long per_block = (64 * 1024) / window_bytes;
+    if (per_block < kWarps) per_block = kWarps;
+    prm.slots_per_block = (int)per_block;
+    const int max_slots = ks.k_max + prm.obs_slots;
+    dim3 grid((max_slots + prm.slots_per_block - 1) / prm.slots_per_block, ks.batch * ks.hkv, n_tensors);
     gather_kv_kernel<<<grid, kThreads, 0, stream>>>(prm);
     count_launches(1);
     return cudaGetLastError();
