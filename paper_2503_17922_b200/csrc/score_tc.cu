@@ -46,7 +46,7 @@ __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
 constexpr int kChunkCap = kTcMaxChunkTiles * kTile + kTcMaxWindow;   // token scores a block may hold
-constexpr int kSyncTickets = 16;                         // sync[0] grid-barrier word, tickets from sync[16]
+constexpr int kSyncTickets = 16;                         // sync[0..1] grid barrier, tickets from sync[16]
 
 struct TcArgs {
     KShape s;
@@ -105,44 +105,47 @@ __device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
     if (lane == 0) mbar_arrive(bar);
 }
 
-// Grid-wide barrier of a cooperative launch (all blocks resident).  One word: arrivals in the low 16
-// bits, generation above; the last arriver clears the count and bumps the generation in one atomic.
-// Bounded: a block that waits longer than two seconds gives up, sets its abort flag and the caller
-// tears the block down.
+// Grid-wide barrier of a cooperative launch (all blocks resident).  sync[0] counts arrivals and only
+// grows during a launch: the barrier number `phase` is passed once n_blocks * phase blocks have
+// arrived (one atomic and one polled word per barrier).  sync[1] counts the blocks that have left
+// the kernel; the last one clears both words for the next launch.  Bounded: a block that waits
+// longer than two seconds gives up, sets its abort flag and the caller tears the block down.
 __device__ __forceinline__ int ld_acquire_gpu(const int *p)
 {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void grid_barrier(int *sync, int n_blocks, volatile int *abort_flag)
+__device__ __forceinline__ void grid_barrier(int *sync, int n_blocks, int phase, volatile int *abort_flag)
 {
     __syncthreads();
     if (threadIdx.x == 0 && !*abort_flag) {
         // the fence of thread 0 is cumulative: it also publishes what the other threads of the block
         // wrote before the block barrier above
         __threadfence();
-        const int old = atomicAdd(sync, 1);
-        if ((old & 0xffff) == n_blocks - 1) {
-            __threadfence();
-            atomicAdd(sync, 0x10000 - n_blocks);
-        } else {
-            const int gen = old >> 16;
-            unsigned long long t0 = 0;
-            for (uint32_t spin = 1; (ld_acquire_gpu(sync) >> 16) == gen; ++spin) {
-                if ((spin & 1023u) == 0u) {
-                    const unsigned long long now = global_timer_ns();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > 2 * kWaitLimitNs) {
-                        *abort_flag = 1;
-                        break;
-                    }
+        atomicAdd(sync, 1);
+        const int target = n_blocks * phase;
+        unsigned long long t0 = 0;
+        for (uint32_t spin = 1; ld_acquire_gpu(sync) < target; ++spin) {
+            if ((spin & 1023u) == 0u) {
+                const unsigned long long now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > 2 * kWaitLimitNs) {
+                    *abort_flag = 1;
+                    break;
                 }
             }
         }
         __threadfence();
     }
     __syncthreads();
+}
+__device__ __forceinline__ void grid_barrier_leave(int *sync, int n_blocks)
+{
+    if (atomicAdd(sync + 1, 1) == n_blocks - 1) {
+        atomicExch(sync, 0);
+        atomicExch(sync + 1, 0);
+    }
 }
 
 // geometry of one work item
@@ -202,11 +205,12 @@ __device__ __forceinline__ void score_accumulate(const float (&v)[N], const floa
     }
 }
 
-// Eq. 4 for one window of compile-time length by one thread: the values sit in registers, the rank
-// of each (value descending, position ascending) comes from omega*omega independent comparisons, and
-// the p best are summed in position order.
+// Eq. 4 for one window of compile-time length by four neighbouring lanes: each keeps the window in
+// registers, ranks a quarter of its values (value descending, position ascending; omega
+// independent comparisons per value) and sums those among the p best; two shuffles add the four
+// partial sums in a fixed order.  Every lane of the warp must call this.
 template <int omega>
-__device__ __forceinline__ float pool_window_regs(const float *w, int size, int p)
+__device__ __forceinline__ float pool_window_quad(const float *w, int size, int p, int part)
 {
     float v[omega];
 #pragma unroll
@@ -214,13 +218,18 @@ __device__ __forceinline__ float pool_window_regs(const float *w, int size, int 
     const int p_eff = p < size ? p : size;
     float acc = 0.f;
 #pragma unroll
-    for (int x = 0; x < omega; ++x) {
+    for (int q4 = 0; q4 < omega / 4; ++q4) {
+        // value number x = 4 * q4 + part: selected with a 4-way choice so that v[] stays in registers
+        const float a0 = v[4 * q4], a1 = v[4 * q4 + 1], a2 = v[4 * q4 + 2], a3 = v[4 * q4 + 3];
+        const float mine = part == 0 ? a0 : (part == 1 ? a1 : (part == 2 ? a2 : a3));
+        const int x = 4 * q4 + part;
         int rank = 0;
 #pragma unroll
-        for (int y = 0; y < omega; ++y)
-            if (y != x) rank += (int)(v[y] > v[x]) | ((int)(v[y] == v[x]) & (int)(y < x));
-        acc += (x < size && rank < p_eff) ? v[x] : 0.f;
+        for (int y = 0; y < omega; ++y) rank += (int)(v[y] > mine) | ((int)(v[y] == mine) & (int)(y < x));
+        acc += (x < size && rank < p_eff) ? mine : 0.f;
     }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
     return acc / (float)p_eff;
 }
 
@@ -302,10 +311,13 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.n_tiles = im.j_end > im.j_begin ? (im.j_end - im.j_begin + kTile - 1) / kTile : 0;
     };
 
-    // Called by every warp except the producer (which has no use for Q and starts streaming keys at
-    // once); ends with a barrier among those warps.  Four loads are in flight per thread.
+    // Called by every warp except the producer; ends with a barrier among those warps.  Four loads
+    // are in flight per thread.  The producer starts streaming key tiles once these small loads
+    // have been ISSUED (go_producer): a tile burst issued first would sit in front of them in the
+    // SM's memory pipeline for microseconds.
     constexpr int kLoaders = kThreads - 32;
-    auto load_q_image = [&](const Item &im) {
+    auto go_producer = [&]() { asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory"); };
+    auto load_q_image = [&](const Item &im, bool signal) {
         if (q_unit_loaded != im.unit) {
             const __nv_bfloat16 *q_unit = q + im.b * s.qsb + (long long)im.h * s.G * s.qsh;
             const int vshift = s.d == 128 ? 4 : 3;            // log2(16-byte vectors per row)
@@ -324,6 +336,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                         }
                     }
                 }
+                if (signal && base == (int)threadIdx.x - 32) go_producer();
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int idx = base + u * kLoaders;
@@ -333,7 +346,10 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                     }
                 }
             }
+            if (signal && (int)threadIdx.x - 32 >= total) go_producer();   // a thread without a share of the image
             fence_proxy_async_smem();
+        } else if (signal) {
+            go_producer();
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
     };
@@ -488,9 +504,10 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 continue;
             }
             if (warp == 0) {
+                asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
                 if (lane == 0) produce(im);
             } else {
-                load_q_image(im);
+                load_q_image(im, true);
                 if (warp == 1) {
                     if (lane == 0) issue_mma(im, false);
                 } else {
@@ -525,7 +542,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             __syncthreads();   // `part` is rewritten by the next item
         }
 
-        grid_barrier(a.sync, gridDim.x, &abort_s);
+        grid_barrier(a.sync, gridDim.x, wave + 1, &abort_s);
         if (abort_s) break;
 
         // ------------------------------------------------------------------ sweep 2 (+ selection)
@@ -544,9 +561,10 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 continue;
             }
             if (warp == 0) {
+                asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
                 if (lane == 0) produce(im);
             } else {
-                load_q_image(im);
+                load_q_image(im, false);
                 // Eq. 1's normaliser of every row: merge the partial statistics of the unit's chunks.
                 // kMergers threads share a row (each takes every kMergers-th chunk), then one of them
                 // merges their results; both steps in a fixed order.
@@ -556,30 +574,31 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 if (tl < kMergers * q_rows) {
                     const int r = tl % q_rows, mp = tl / q_rows;
                     float M = -INFINITY, sum = 0.f;
-                    if (r < s.R) {
-                        const int len1 = tc_chunk_len(im.n, cpu, 1);
-                        const int used = (im.n + len1 - 1) / len1;
-                        const float2 *st = a.stats + (size_t)im.unit * a.n_stat_chunks * a.r_pad + r;
-                        for (int c0 = mp; c0 < used; c0 += 8 * kMergers) {
-                            float2 p[8];
+                    const int len1 = tc_chunk_len(im.n, cpu, 1);
+                    const int used = r < s.R ? (im.n + len1 - 1) / len1 : 0;
+                    const float2 *st = a.stats + (size_t)im.unit * a.n_stat_chunks * a.r_pad + r;
+                    for (int c0 = mp; c0 < used || c0 == mp; c0 += 8 * kMergers) {
+                        float2 p[8];
 #pragma unroll
-                            for (int u = 0; u < 8; ++u) {
-                                const int cidx = c0 + u * kMergers;
-                                p[u] = cidx < used ? __ldcg(st + (size_t)cidx * a.r_pad) : make_float2(-INFINITY, 0.f);
-                            }
-                            float Mn = M;
+                        for (int u = 0; u < 8; ++u) {
+                            const int cidx = c0 + u * kMergers;
+                            p[u] = cidx < used ? __ldcg(st + (size_t)cidx * a.r_pad) : make_float2(-INFINITY, 0.f);
+                        }
+                        if (c0 == mp) go_producer();   // this thread's first loads are on their way
+                        float Mn = M;
 #pragma unroll
-                            for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, p[u].x);
-                            if (Mn > -INFINITY) {
-                                sum *= fast_exp2(M - Mn);
+                        for (int u = 0; u < 8; ++u) Mn = fmaxf(Mn, p[u].x);
+                        if (Mn > -INFINITY) {
+                            sum *= fast_exp2(M - Mn);
 #pragma unroll
-                                for (int u = 0; u < 8; ++u)
-                                    if (p[u].y > 0.f) sum += p[u].y * fast_exp2(p[u].x - Mn);
-                                M = Mn;
-                            }
+                            for (int u = 0; u < 8; ++u)
+                                if (p[u].y > 0.f) sum += p[u].y * fast_exp2(p[u].x - Mn);
+                            M = Mn;
                         }
                     }
                     merged[mp * q_rows + r] = make_float2(M, sum);
+                } else {
+                    go_producer();
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
                 if (tl < 256) {
@@ -618,14 +637,17 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 float *ws_out = a.window_scores + (size_t)im.unit * s.kw_max + im.j_begin / s.omega;
                 const int n_win = (n_tok + s.omega - 1) / s.omega;
                 if (s.omega == 16 || s.omega == 8 || s.omega == 32 || s.omega == 4) {
-                    for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
-                        const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
+                    const int part = threadIdx.x & 3;
+                    for (int lw0 = 0; lw0 < n_win; lw0 += kThreads / 4) {      // uniform trip count: shuffles inside
+                        const int lw = lw0 + (threadIdx.x >> 2);
+                        const bool live = lw < n_win;
+                        const int lo = live ? lw * s.omega : 0, size = live ? min(s.omega, n_tok - lo) : 1;
                         float r;
-                        if (s.omega == 16) r = pool_window_regs<16>(t_chunk + lo, size, s.p);
-                        else if (s.omega == 8) r = pool_window_regs<8>(t_chunk + lo, size, s.p);
-                        else if (s.omega == 32) r = pool_window_regs<32>(t_chunk + lo, size, s.p);
-                        else r = pool_window_regs<4>(t_chunk + lo, size, s.p);
-                        ws_out[lw] = r;
+                        if (s.omega == 16) r = pool_window_quad<16>(t_chunk + lo, size, s.p, part);
+                        else if (s.omega == 8) r = pool_window_quad<8>(t_chunk + lo, size, s.p, part);
+                        else if (s.omega == 32) r = pool_window_quad<32>(t_chunk + lo, size, s.p, part);
+                        else r = pool_window_quad<4>(t_chunk + lo, size, s.p, part);
+                        if (live && part == 0) ws_out[lw] = r;
                     }
                 }
                 else {
@@ -676,6 +698,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             }
         }
         if (abort_s) atomicOr(a.status, kStatusWaitExpired);
+        else grid_barrier_leave(a.sync, gridDim.x);
     }
     tc_fence_before_sync();
     __syncthreads();
