@@ -275,6 +275,54 @@ def wkv_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_out_la
                                     workspace.numel(), _stream(stream)), "wkv_compress_group")
 
 
+class PreparedCall:
+    """A C-ABI call with its arguments marshalled once (pointer tables, shape, stream): `run()` is a
+    single foreign call, so that a loop over many groups is not bound by Python."""
+
+    def __init__(self, fn, what: str, args: tuple, keep: tuple):
+        self._fn, self._what, self._args, self._keep = fn, what, args, keep
+
+    def run(self) -> None:
+        st = self._fn(*self._args)
+        if st != 0:
+            _check(st, self._what)
+
+
+def prepare_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers,
+                           window_scores, window_idx, kept_len, workspace, cu_seqlens_out=None,
+                           keep_capacity: int = 0, stream=None) -> PreparedCall:
+    arrs = (_ptr_array(k_layers), _ptr_array(v_layers), _ptr_array(k_out_layers), _ptr_array(v_out_layers))
+    args = (ctypes.byref(prob.shape), len(k_layers), _ptr(q_obs_leader), arrs[0], arrs[1], arrs[2], arrs[3],
+            _ptr(window_scores), _ptr(window_idx), _ptr(kept_len), _ptr(cu_seqlens_out), keep_capacity,
+            _ptr(workspace), workspace.numel(), _stream(stream))
+    return PreparedCall(lib().wkv_compress_group, "wkv_compress_group", args,
+                        (prob, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers, window_scores,
+                         window_idx, kept_len, workspace, cu_seqlens_out, arrs))
+
+
+def prepare_score_windows(prob: Problem, q_obs, k_leader, window_scores, token_scores, workspace,
+                          stream=None) -> PreparedCall:
+    args = (ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader), _ptr(window_scores), _ptr(token_scores),
+            _ptr(workspace), workspace.numel(), _stream(stream))
+    return PreparedCall(lib().wkv_score_windows, "wkv_score_windows", args,
+                        (prob, q_obs, k_leader, window_scores, token_scores, workspace))
+
+
+def prepare_select_topk_windows(prob: Problem, window_scores, window_idx, kept_len, stream=None) -> PreparedCall:
+    args = (ctypes.byref(prob.shape), _ptr(window_scores), _ptr(window_idx), _ptr(kept_len), _stream(stream))
+    return PreparedCall(lib().wkv_select_topk_windows, "wkv_select_topk_windows", args,
+                        (prob, window_scores, window_idx, kept_len))
+
+
+def prepare_gather_kv(prob: Problem, k_layers, v_layers, window_idx, k_out_layers, v_out_layers,
+                      cu_seqlens_out=None, keep_capacity: int = 0, stream=None) -> PreparedCall:
+    arrs = (_ptr_array(k_layers), _ptr_array(v_layers), _ptr_array(k_out_layers), _ptr_array(v_out_layers))
+    args = (ctypes.byref(prob.shape), len(k_layers), arrs[0], arrs[1], _ptr(window_idx), arrs[2], arrs[3],
+            _ptr(cu_seqlens_out), keep_capacity, _stream(stream))
+    return PreparedCall(lib().wkv_gather_kv, "wkv_gather_kv", args,
+                        (prob, k_layers, v_layers, window_idx, k_out_layers, v_out_layers, cu_seqlens_out, arrs))
+
+
 def wkv_compress_group_host(prob: Problem, q_obs_host, k_layers_host, v_layers_host, k_out_host, v_out_host,
                             window_idx_host, kept_len_host, q_obs_dev, k_layers_dev, v_layers_dev,
                             k_out_dev, v_out_dev, window_idx_dev, kept_len_dev, keep_capacity, workspace,
