@@ -205,31 +205,34 @@ __device__ __forceinline__ void score_accumulate(const float (&v)[N], const floa
     }
 }
 
-// Eq. 4 for one window of compile-time length by four neighbouring lanes: each keeps the window in
-// registers, ranks a quarter of its values (value descending, position ascending; omega
-// independent comparisons per value) and sums those among the p best; two shuffles add the four
-// partial sums in a fixed order.  Every lane of the warp must call this.
+// Eq. 4 for one window of compile-time length (a power of two) by one thread: a bitonic sorting
+// network in registers (every compare-exchange of a stage is independent of the others, so the
+// thread is not latency-bound), then the p largest are summed in descending order.  Positions
+// beyond `size` (ragged last window) hold -inf and sort to the end.
 template <int omega>
-__device__ __forceinline__ float pool_window_quad(const float *w, int size, int p, int part)
+__device__ __forceinline__ float pool_window_sorted(const float *w, int size, int p)
 {
     float v[omega];
 #pragma unroll
     for (int x = 0; x < omega; ++x) v[x] = x < size ? w[x] : -INFINITY;
+#pragma unroll
+    for (int k = 2; k <= omega; k <<= 1)
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+            for (int i = 0; i < omega; ++i) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const float hi = fmaxf(v[i], v[l]), lo = fminf(v[i], v[l]);
+                    const bool descending = (i & k) == 0;
+                    v[i] = descending ? hi : lo;
+                    v[l] = descending ? lo : hi;
+                }
+            }
     const int p_eff = p < size ? p : size;
     float acc = 0.f;
 #pragma unroll
-    for (int q4 = 0; q4 < omega / 4; ++q4) {
-        // value number x = 4 * q4 + part: selected with a 4-way choice so that v[] stays in registers
-        const float a0 = v[4 * q4], a1 = v[4 * q4 + 1], a2 = v[4 * q4 + 2], a3 = v[4 * q4 + 3];
-        const float mine = part == 0 ? a0 : (part == 1 ? a1 : (part == 2 ? a2 : a3));
-        const int x = 4 * q4 + part;
-        int rank = 0;
-#pragma unroll
-        for (int y = 0; y < omega; ++y) rank += (int)(v[y] > mine) | ((int)(v[y] == mine) & (int)(y < x));
-        acc += (x < size && rank < p_eff) ? mine : 0.f;
-    }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    for (int x = 0; x < omega; ++x) acc += x < p_eff ? v[x] : 0.f;
     return acc / (float)p_eff;
 }
 
@@ -565,12 +568,19 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 if (lane == 0) produce(im);
             } else {
                 load_q_image(im, false);
+                if (warp == 1) {
+                    // the MMAs do not need the normalisers: the first accumulators fill while the
+                    // compute warps merge the statistics
+                    go_producer();
+                    if (lane == 0) issue_mma(im, true);
+                } else {
                 // Eq. 1's normaliser of every row: merge the partial statistics of the unit's chunks.
                 // kMergers threads share a row (each takes every kMergers-th chunk), then one of them
                 // merges their results; both steps in a fixed order.
-                constexpr int kMergers = kLoaders / q_rows;
+                constexpr int kComputeThreads = kThreads - 64;
+                constexpr int kMergers = kComputeThreads / q_rows;
                 float2 *merged = &part[0][0][0];
-                const int tl = threadIdx.x - 32;
+                const int tl = threadIdx.x - 64;
                 if (tl < kMergers * q_rows) {
                     const int r = tl % q_rows, mp = tl / q_rows;
                     float M = -INFINITY, sum = 0.f;
@@ -600,7 +610,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 } else {
                     go_producer();
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
+                asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
                 if (tl < 256) {
                     float v = -INFINITY;
                     if (tl < s.R) {
@@ -618,11 +628,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                     }
                     neg_lse2[tl] = v;
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(kLoaders) : "memory");
-                if (warp == 1) {
-                    if (lane == 0) issue_mma(im, true);
-                } else {
-                    compute_scores(im);
+                asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
+                compute_scores(im);
                 }
             }
             q_unit_loaded = im.unit;
@@ -637,17 +644,16 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 float *ws_out = a.window_scores + (size_t)im.unit * s.kw_max + im.j_begin / s.omega;
                 const int n_win = (n_tok + s.omega - 1) / s.omega;
                 if (s.omega == 16 || s.omega == 8 || s.omega == 32 || s.omega == 4) {
-                    const int part = threadIdx.x & 3;
-                    for (int lw0 = 0; lw0 < n_win; lw0 += kThreads / 4) {      // uniform trip count: shuffles inside
-                        const int lw = lw0 + (threadIdx.x >> 2);
-                        const bool live = lw < n_win;
-                        const int lo = live ? lw * s.omega : 0, size = live ? min(s.omega, n_tok - lo) : 1;
+                    // consecutive windows go to different warps so that all four schedulers take part
+                    for (int i = threadIdx.x; i < n_win; i += kThreads) {
+                        const int lw = i;
+                        const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
                         float r;
-                        if (s.omega == 16) r = pool_window_quad<16>(t_chunk + lo, size, s.p, part);
-                        else if (s.omega == 8) r = pool_window_quad<8>(t_chunk + lo, size, s.p, part);
-                        else if (s.omega == 32) r = pool_window_quad<32>(t_chunk + lo, size, s.p, part);
-                        else r = pool_window_quad<4>(t_chunk + lo, size, s.p, part);
-                        if (live && part == 0) ws_out[lw] = r;
+                        if (s.omega == 16) r = pool_window_sorted<16>(t_chunk + lo, size, s.p);
+                        else if (s.omega == 8) r = pool_window_sorted<8>(t_chunk + lo, size, s.p);
+                        else if (s.omega == 32) r = pool_window_sorted<32>(t_chunk + lo, size, s.p);
+                        else r = pool_window_sorted<4>(t_chunk + lo, size, s.p);
+                        ws_out[lw] = r;
                     }
                 }
                 else {
