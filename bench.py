@@ -180,15 +180,12 @@ def main() -> None:
         return
 
     import torch
-    import torch.distributed as dist
-    from paper_2503_17922_b200 import binding
+    from paper_2503_17922_b200 import binding, replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    # replicas only: every rank runs the whole path on its own copy of the workload (no exchange step)
+    rank, world, local = replicas.rank_env()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init("nccl", torch.device("cuda", local))
     binding.lib()          # fails loudly if the CUDA library is missing
 
     w = pick_workload(args.workload)
@@ -230,10 +227,7 @@ def main() -> None:
     gather_calls = [binding.prepare_gather_kv(prob, d["k"], d["v"], out["window_idx"], out["k_out"], out["v_out"],
                                               keep_capacity=cap, stream=stream) for d in dev_groups]
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    barrier = replicas.barrier
 
     with torch.cuda.stream(stream):
         for i in range(warmup):
@@ -265,12 +259,9 @@ def main() -> None:
             ms_total = sum(a.elapsed_time(b) for a, b in evs)
         launches = binding.wkv_launch_count() - launches0
         clocks = sampler.stop() if rank == 0 else None
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+        ms_total = replicas.max_over_ranks(ms_total, "cuda")
         ms_per_step = ms_total / args.steps
-        value = tokens * world / (ms_per_step * 1e-3)
+        value = replicas.whole_job_rate(tokens, world, ms_per_step)
         if binding.device_status(work) != 0:
             raise RuntimeError("a kernel reported an expired wait: results invalid")
 
@@ -361,13 +352,11 @@ def main() -> None:
             e2e_step(i)
         barrier()
         dt = time.perf_counter() - t0
-        tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt = replicas.max_over_ranks(dt, "cuda")
         nb = lambda t: t.numel() * t.element_size()
         h2d = nb(hsets[0]["q"]) + sum(nb(x) for x in hsets[0]["k"] + hsets[0]["v"])
         d2h = sum(nb(x) for x in h_k_out + h_v_out) + nb(h_idx) + nb(h_kept)
-        e2e = {"value": tokens * world * e2e_steps / float(tt.item()), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": tokens * world * e2e_steps / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
     # ---- the oracle on the host cores (rank 0, single-GPU runs only)
@@ -396,8 +385,7 @@ def main() -> None:
                           "score_only": ms_score, "select_standalone": ms_select, "gather": ms_gather},
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "clocks": clocks,
         }))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 if __name__ == "__main__":

@@ -98,6 +98,21 @@ int32_t wkv_kw_max(const wkv_shape *s);   /* max_b K_w,b, at least 1 */
 int32_t wkv_k_max(const wkv_shape *s);    /* max_b k_b,   at least 1 */
 int32_t wkv_keep_max(const wkv_shape *s); /* max_b (k_b*omega + min(alpha, n_b)): row capacity of the dense compact cache */
 
+/*
+ * Dynamic (pyramid) budget allocation, Eq. 5-7: the H = n_layers / gamma groups get budgets in an
+ * arithmetic sequence from b^0 (bottom group) down to b^{H-1} = b_total / (lambda * H) (top group),
+ * b^0 = 2 * b_total / H - b^{H-1}, and each group's budget is split evenly over its gamma layers.
+ * lambda = lambda_num / lambda_den (the paper uses 14) is taken as a ratio of integers so that the
+ * result is exact: out[h] = floor(b^h / gamma) tokens per layer of group h, and the tokens lost to
+ * the flooring go, in whole multiples of gamma, to group 0.  The per-layer values are what the
+ * `budget` / `budgets_host` fields of wkv_shape expect.  Host function, no device work.
+ *   b_total         total budget over all layers (e.g. n_layers * average per-layer budget)
+ *   per_layer_out   HOST out, int32 [n_layers / gamma]
+ * Returns WKV_ERR_SHAPE for n_layers % gamma != 0, lambda < 1 or non-positive sizes.
+ */
+int wkv_group_budgets(int32_t n_layers, int32_t gamma, int64_t b_total, int32_t lambda_num, int32_t lambda_den,
+                      int32_t *per_layer_out);
+
 /* Bytes of DEVICE scratch that wkv_score_windows / wkv_compress_group need for this
  * shape (256-byte aligned base expected).  Returns 0 for an invalid shape. */
 size_t wkv_workspace_bytes(const wkv_shape *s);

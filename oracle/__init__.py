@@ -206,6 +206,25 @@ def gather_layer(src: np.ndarray, window_idx: np.ndarray, *, n_kv_heads: int, l_
     return dst
 
 
+def group_budgets(n_layers: int, gamma: int, b_total: int, lam) -> Dict[str, object]:
+    """Eq. 5-7 in exact rational arithmetic.  Returns the real-valued group budgets b^h (Fractions),
+    the real-valued per-layer budgets b^h / gamma, and the integer per-layer budgets: floor, with
+    the tokens lost to the flooring given to group 0 in whole multiples of gamma."""
+    from fractions import Fraction
+    H = n_layers // gamma
+    T, lam = Fraction(b_total), Fraction(lam)
+    if H == 1:
+        b = [T]
+    else:
+        b_top = T / (lam * H)                      # Eq. 6, top group
+        b_bottom = 2 * T / H - b_top               # Eq. 6, bottom group
+        b = [b_bottom - (b_bottom - b_top) / (H - 1) * h for h in range(H)]   # Eq. 7
+    per_layer = [x / gamma for x in b]
+    ints = [int(x // 1) for x in per_layer]
+    ints[0] += (b_total - gamma * sum(ints)) // gamma
+    return {"group": b, "per_layer": per_layer, "per_layer_int": ints}
+
+
 def keep_max(seqlens: Sequence[int], budgets: Sequence[int], l_obs: int, window: int) -> int:
     """Row capacity of the dense compact cache: max over sequences of k*omega + min(alpha, n)."""
     return max(num_selected(int(n), l_obs, window, int(b)) * window + min(l_obs, int(n))

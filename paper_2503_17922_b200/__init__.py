@@ -5,4 +5,4 @@
 `workloads` seeded synthetic inputs of the benchmark configurations.
 `build`     compiles the library in-tree with nvcc.
 """
-__all__ = ["binding", "workloads", "build"]
+__all__ = ["binding", "workloads", "build", "replicas"]

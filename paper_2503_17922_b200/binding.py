@@ -22,7 +22,7 @@ WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05 = 0, 1, 2
 WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
-    "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max",
+    "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
     for name in ("wkv_kw_max", "wkv_k_max", "wkv_keep_max"):
         getattr(L, name).restype = i32
         getattr(L, name).argtypes = [sp]
+    L.wkv_group_budgets.restype = ctypes.c_int
+    L.wkv_group_budgets.argtypes = [i32, i32, ctypes.c_int64, i32, i32, vp]
     L.wkv_workspace_bytes.restype = sz
     L.wkv_workspace_bytes.argtypes = [sp]
     L.wkv_score_windows.restype = ctypes.c_int
@@ -342,6 +344,14 @@ def wkv_compress_group_host(prob: Problem, q_obs_host, k_layers_host, v_layers_h
 def device_status(workspace) -> int:
     """The workspace's status word (synchronises): 0, or the OR of the error bits a kernel has set."""
     return int(workspace[:4].view(__import__("torch").int32).item())
+
+
+def wkv_group_budgets(n_layers: int, gamma: int, b_total: int, lambda_num: int = 14, lambda_den: int = 1) -> np.ndarray:
+    """Eq. 5-7: per-layer budget of each of the n_layers / gamma groups (host arithmetic, exact)."""
+    out = np.zeros(max(n_layers // max(gamma, 1), 1), dtype=np.int32)
+    _check(lib().wkv_group_budgets(n_layers, gamma, b_total, lambda_num, lambda_den, out.ctypes.data),
+           "wkv_group_budgets")
+    return out
 
 
 def wkv_launch_count() -> int:

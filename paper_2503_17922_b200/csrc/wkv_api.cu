@@ -309,6 +309,38 @@ int32_t wkv_keep_max(const wkv_shape *s)
     return resolve(s, ks) == WKV_OK ? keep_max_of(s) : 0;
 }
 
+int wkv_group_budgets(int32_t n_layers, int32_t gamma, int64_t b_total, int32_t lambda_num, int32_t lambda_den,
+                      int32_t *per_layer_out)
+{
+    if (!per_layer_out) {
+        set_error_detail("per_layer_out is NULL");
+        return WKV_ERR_NULL;
+    }
+    if (n_layers < 1 || gamma < 1 || n_layers % gamma || b_total < 0 || lambda_den < 1 || lambda_num < lambda_den) {
+        set_error_detail("group budgets: n_layers %d, gamma %d, b_total %lld, lambda %d/%d", n_layers, gamma,
+                         (long long)b_total, lambda_num, lambda_den);
+        return WKV_ERR_SHAPE;
+    }
+    const int H = n_layers / gamma;
+    if (H == 1) {
+        per_layer_out[0] = (int32_t)(b_total / gamma);
+        return WKV_OK;
+    }
+    // b^h = T * [(2 num - den)(H - 1) - 2 (num - den) h] / (num * H * (H - 1))   (Eq. 6 into Eq. 7)
+    typedef __int128 wide;
+    const wide T = b_total, num = lambda_num, den = lambda_den;
+    const wide denom = num * H * (H - 1) * gamma;
+    wide used = 0;
+    for (int h = 0; h < H; ++h) {
+        const wide numer = T * ((2 * num - den) * (H - 1) - 2 * (num - den) * h);
+        const wide per_layer = numer / denom;     // numer >= 0 because lambda >= 1
+        per_layer_out[h] = (int32_t)per_layer;
+        used += per_layer * gamma;
+    }
+    per_layer_out[0] += (int32_t)((T - used) / gamma);
+    return WKV_OK;
+}
+
 size_t wkv_workspace_bytes(const wkv_shape *s)
 {
     KShape ks;

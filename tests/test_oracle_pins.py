@@ -317,3 +317,41 @@ def test_workload_shapes_match_the_configs():
     back = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x))
     tx = torch.from_numpy(x).to(torch.bfloat16).float().numpy()      # library rounding
     np.testing.assert_array_equal(back, tx)
+
+
+# ------------------------------------------------------------------ Eq. 5-7: pyramid budgets
+def test_group_budgets_closed_forms():
+    from fractions import Fraction
+    # the configuration of the paper's main experiments: 32 layers, groups of 8, lambda = 14, and an
+    # average of 2048 tokens per layer.  Hand-derived from Eq. 6-7: b^3 = 65536/56, b^0 = 32768 - b^3.
+    r = oracle.group_budgets(32, 8, 32 * 2048, 14)
+    assert r["group"][3] == Fraction(65536, 56) and r["group"][0] == Fraction(32768) - Fraction(65536, 56)
+    assert [round(float(x), 1) for x in r["per_layer"]] == [3949.7, 2681.9, 1414.1, 146.3]
+    for n_layers, gamma, total, lam in [(32, 8, 65536, 14), (28, 7, 28 * 512, 14), (32, 4, 32 * 1024, Fraction(7, 2)),
+                                        (32, 1, 32 * 2048, 14), (8, 8, 4096, 14)]:
+        r = oracle.group_budgets(n_layers, gamma, total, lam)
+        b, H = r["group"], n_layers // gamma
+        assert sum(b) == total                                            # Eq. 5
+        if H > 1:
+            assert b[-1] * lam * H == total                               # Eq. 6
+            assert len({b[h] - b[h + 1] for h in range(H - 1)}) == 1      # Eq. 7: arithmetic sequence
+            assert b[0] >= b[-1]
+        ints = r["per_layer_int"]
+        assert 0 <= total - gamma * sum(ints) < gamma                     # nothing above the budget, < gamma lost
+        assert all(ints[h] == int(r["per_layer"][h]) for h in range(1, H))
+
+
+def test_group_budgets_library_matches_oracle():
+    from fractions import Fraction
+    from paper_2503_17922_b200 import binding, build
+    build.build_library()
+    for n_layers, gamma, total, num, den in [(32, 8, 65536, 14, 1), (28, 7, 14336, 14, 1), (32, 4, 32768, 7, 2),
+                                             (32, 1, 65536, 14, 1), (8, 8, 4096, 14, 1), (32, 8, 12345, 3, 1),
+                                             (64, 4, 10 ** 9, 14, 1), (32, 8, 0, 14, 1), (32, 8, 100, 1, 1)]:
+        got = binding.wkv_group_budgets(n_layers, gamma, total, num, den)
+        exp = oracle.group_budgets(n_layers, gamma, total, Fraction(num, den))["per_layer_int"]
+        assert got.tolist() == exp, (n_layers, gamma, total, num, den)
+    with pytest.raises(binding.WkvError):
+        binding.wkv_group_budgets(30, 8, 1000)
+    with pytest.raises(binding.WkvError):
+        binding.wkv_group_budgets(32, 8, 1000, 1, 2)      # lambda < 1

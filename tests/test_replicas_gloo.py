@@ -1,0 +1,54 @@
+"""The benchmark's N > 1 path on CPU: two gloo ranks run the replica plumbing (barrier, maximum of
+the per-rank times, whole-job rate) exactly as bench.py does over NCCL."""
+import os
+import socket
+import sys
+
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank: int, world: int, port: int, out_dir: str) -> None:
+    sys.path.insert(0, ROOT)
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    from paper_2503_17922_b200 import replicas
+    assert replicas.rank_env() == (rank, world, rank)
+    replicas.init("gloo")
+    replicas.barrier(sync_cuda=False)
+    my_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow replica
+    total_ms = replicas.max_over_ranks(my_ms)
+    rate = replicas.whole_job_rate(32768, world, total_ms / 4)
+    replicas.barrier(sync_cuda=False)
+    with open(os.path.join(out_dir, f"rank{rank}.txt"), "w") as f:
+        f.write(f"{total_ms} {rate}")
+    replicas.shutdown()
+
+
+def test_two_gloo_ranks_agree_on_the_slowest_time(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    results = [open(tmp_path / f"rank{r}.txt").read().split() for r in range(world)]
+    for total_ms, rate in results:
+        assert float(total_ms) == 15.0                                   # the maximum over the ranks
+        assert abs(float(rate) - 32768 * 2 / (15.0 / 4 * 1e-3)) < 1e-6   # both replicas count
+
+
+def test_single_process_is_a_noop():
+    sys.path.insert(0, ROOT)
+    from paper_2503_17922_b200 import replicas
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+        os.environ.pop(k, None)
+    assert replicas.rank_env() == (0, 1, 0)
+    replicas.init("gloo")
+    assert replicas.max_over_ranks(3.5) == 3.5
+    assert replicas.whole_job_rate(100, 1, 1.0) == 100000.0
