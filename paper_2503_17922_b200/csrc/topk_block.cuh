@@ -1,8 +1,8 @@
 // Budgeted window selection (sentence after Eq. 4) for one unit by one thread block: the k-th
-// largest window score is found with a 4-pass, 8-bit radix select over an order-preserving
-// integer image of the fp32 scores, then the selected window indices are emitted in ascending
-// order with block-wide prefix sums.  Equal scores at the threshold go to the lower window
-// index.  Integer arithmetic only after the key mapping, so the result is exact and
+// largest window score is found with a 3-pass radix select (11 + 11 + 10 bits) over an
+// order-preserving integer image of the fp32 scores, then the selected window indices are emitted
+// in ascending order with one block-wide prefix sum.  Equal scores at the threshold go to the
+// lower window index.  Integer arithmetic only after the key mapping, so the result is exact and
 // deterministic.  Used by the stand-alone selection kernel and by the fused score kernel.
 #pragma once
 
@@ -10,9 +10,11 @@
 
 namespace wkv {
 
+constexpr int kTopkBins = 2048;
+
 struct TopkSmem {
-    int hist[256];
-    int warp_sums[32];
+    __align__(16) int hist[kTopkBins];
+    int warp_sums[33];
     unsigned prefix;
     int remaining;
     int last_selected;
@@ -26,7 +28,9 @@ __device__ __forceinline__ unsigned topk_order_key(float f)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// exclusive prefix sum of `v` over the NT threads of the block; also returns the total
+// exclusive prefix sum of `v` over the NT threads of the block; also returns the total.  Shared
+// memory is one pipe for the whole SM, so the scan touches it as little as possible: one word
+// written per warp, the warp totals scanned by warp 0 with shuffles, two words read per thread.
 template <int NT>
 __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total)
 {
@@ -41,29 +45,38 @@ __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total
     __syncthreads();   // protects warp_sums from the previous use
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    int base = 0, tot = 0;
+    if (warp == 0) {
+        const int mine = lane < kWarps ? warp_sums[lane] : 0;
+        int w_incl = mine;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        int x = warp_sums[w];
-        if (w < warp) base += x;
-        tot += x;
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, w_incl, o);
+            if (lane >= o) w_incl += t;
+        }
+        if (lane < kWarps) warp_sums[lane] = w_incl - mine;       // exclusive base of warp `lane`
+        if (lane == 31) warp_sums[32] = w_incl;                    // grand total
     }
-    total = tot;
-    return base + incl - v;
+    __syncthreads();
+    total = warp_sums[32];
+    return warp_sums[warp] + incl - v;
 }
 
 // All NT threads of the block call this.  `sc` are the unit's kw window scores (read through L2,
 // so scores written by other blocks of the same grid are seen once the caller has synchronised
 // with them), `out` receives k ascending indices followed by -1 up to k_max.
 // Thread t owns the windows [t*E, (t+1)*E), E = ceil(kw / NT).  With E <= kTopkRegs the keys are
-// read once and stay in registers through the four radix passes and the compaction (one trip to
-// L2 instead of six); longer lists are re-read.
-constexpr int kTopkRegs = 8;
+// read once and stay in registers through the radix passes and the compaction (one trip to L2
+// instead of five); longer lists are re-read.
+constexpr int kTopkRegs = 4;
 
 template <int NT, bool IN_REGS>
 __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, int kw, int k, int *out,
                                                  int *kept_len_out, int n, int alpha, int omega, int obs_rows)
 {
+    // the histogram is scanned by `kScanners` threads (a power of two), kBinsPer bins each
+    constexpr int kScanners = NT >= 512 ? 512 : 256;
+    constexpr int kBinsPer = kTopkBins / kScanners;
+    static_assert(NT >= 256, "block size");
     const int E = (kw + NT - 1) / NT;
     const int w_lo = min(kw, (int)threadIdx.x * E), w_hi = min(kw, w_lo + E);
     unsigned keys[kTopkRegs];
@@ -79,65 +92,67 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
         sm.remaining = k;
         sm.last_selected = 0;
     }
-    for (int x = threadIdx.x; x < 256; x += NT) sm.hist[x] = 0;
+    for (int x = threadIdx.x; x < kTopkBins; x += NT) sm.hist[x] = 0;
     __syncthreads();
     unsigned mask = 0u;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const unsigned digit_mask = pass == 2 ? 1023u : 2047u;
         const unsigned prefix = sm.prefix;
         const int remaining = sm.remaining;
-        // window scores share sign and exponent, so most keys of a pass fall into very few bins:
-        // the lanes of a warp that hit the same bin are counted by one of them
 #pragma unroll
         for (int e = 0; e < (IN_REGS ? kTopkRegs : E); ++e) {
             if (IN_REGS && e >= E) break;   // uniform: E is the same for every thread
-            unsigned bin = 256u;            // not taking part in this pass
+            unsigned bin = kTopkBins;       // not taking part in this pass
             if (w_lo + e < w_hi) {
                 const unsigned key = key_at(e);
-                if ((key & mask) == prefix) bin = (key >> shift) & 0xffu;
+                if ((key & mask) == prefix) bin = (key >> shift) & digit_mask;
             }
+            // window scores share sign and exponent, so the keys of a warp often fall into one bin:
             // the lanes that share the bin of the first participating lane are counted by that lane
-            const unsigned part = __ballot_sync(0xffffffffu, bin < 256u);
+            const unsigned part = __ballot_sync(0xffffffffu, bin < kTopkBins);
             if (part) {
                 const int leader = __ffs(part) - 1;
                 const unsigned pivot = __shfl_sync(0xffffffffu, bin, leader);
                 const unsigned same = __ballot_sync(0xffffffffu, bin == pivot);
                 if ((int)(threadIdx.x & 31) == leader) atomicAdd(&sm.hist[pivot], __popc(same));
-                else if (bin < 256u && bin != pivot) atomicAdd(&sm.hist[bin], 1);
+                else if (bin < kTopkBins && bin != pivot) atomicAdd(&sm.hist[bin], 1);
             }
         }
         __syncthreads();
-        if (threadIdx.x < 32) {
-            // warp 0: the bin (scanning from the top) in which the count reaches `remaining`
-            const int lane = threadIdx.x;
-            int c[8], tot = 0;
+        // the bin (scanning from the top) in which the count reaches `remaining`
+        int c[kBinsPer], mine = 0;
+        if (threadIdx.x < kScanners) {
+            int4 *hv = reinterpret_cast<int4 *>(sm.hist + threadIdx.x * kBinsPer);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                c[i] = sm.hist[lane * 8 + i];
-                sm.hist[lane * 8 + i] = 0;   // ready for the next pass (and the next call)
-                tot += c[i];
-            }
-            int incl = tot;   // inclusive suffix sum over the lanes (lane 31 holds the top bins)
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int t = __shfl_down_sync(0xffffffffu, incl, o);
-                if (lane + o < 32) incl += t;
-            }
-            const int above = incl - tot;
-            if (above < remaining && remaining <= incl) {
-                int rem = remaining - above, bin = lane * 8;
-#pragma unroll
-                for (int i = 7; i >= 0; --i) {
-                    if (c[i] >= rem) {
-                        bin = lane * 8 + i;
-                        break;
-                    }
-                    rem -= c[i];
-                }
-                sm.prefix = prefix | ((unsigned)bin << shift);
-                sm.remaining = rem;   // after the last pass: how many keys equal to the threshold are taken
+            for (int i = 0; i < kBinsPer; i += 4) {
+                const int4 x = hv[i / 4];
+                hv[i / 4] = make_int4(0, 0, 0, 0);   // ready for the next pass
+                c[i] = x.x;
+                c[i + 1] = x.y;
+                c[i + 2] = x.z;
+                c[i + 3] = x.w;
+                mine += (x.x + x.y) + (x.z + x.w);
             }
         }
-        mask |= 0xffu << shift;
+        int total;
+        const int below = topk_block_scan<NT>(mine, sm.warp_sums, total);   // keys in lower bins
+        const int above = total - below - mine;
+        if (threadIdx.x < kScanners && above < remaining && remaining <= above + mine) {
+            int rem = remaining - above, bin = threadIdx.x * kBinsPer;
+#pragma unroll
+            for (int i = kBinsPer - 1; i >= 0; --i) {
+                if (c[i] >= rem) {
+                    bin = threadIdx.x * kBinsPer + i;
+                    break;
+                }
+                rem -= c[i];
+            }
+            sm.prefix = prefix | ((unsigned)bin << shift);
+            sm.remaining = rem;   // after the last pass: how many keys equal to the threshold are taken
+        }
+        mask |= digit_mask << shift;
         __syncthreads();
     }
     const unsigned thr = sm.prefix;
