@@ -62,7 +62,8 @@ def peaks() -> dict:
 def ncu_traffic(kernel: str):
     p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if os.path.exists(p):
-        return json.load(open(p)).get(kernel)
+        v = json.load(open(p)).get(kernel)
+        return v if isinstance(v, (int, float)) else None
     return None
 
 
