@@ -60,10 +60,13 @@ def peaks() -> dict:
 
 
 def ncu_traffic(kernel: str):
-    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    """DRAM bytes per launch of the kernel from the committed ncu capture (config 3 only), or None."""
+    p = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
     if os.path.exists(p):
-        v = json.load(open(p)).get(kernel)
-        return v if isinstance(v, (int, float)) else None
+        for line in open(p):
+            f = line.split()
+            if len(f) == 2 and f[0] == kernel:
+                return int(f[1])
     return None
 
 
@@ -316,7 +319,7 @@ def main() -> None:
     kernel_name = "gather_kv_kernel" if dominant == "gather" else "score_windows_tc (both sweeps + selection)"
     roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": pk["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
-                "traffic": ncu_traffic(dominant), "algorithmic_bytes_per_launch": alg[dominant],
+                "traffic": ncu_traffic(dominant) if args.workload == "C3" else None, "algorithmic_bytes_per_launch": alg[dominant],
                 "launch_ms": dom_ms,
                 "other_kernel": {"kernel": "gather_kv_kernel" if dominant == "score" else "score_windows_tc",
                                  "launch_ms": ms_gather if dominant == "score" else ms_score_select,
