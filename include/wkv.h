@@ -128,10 +128,12 @@ size_t wkv_workspace_bytes(const wkv_shape *s);
  *   k_leader       DEVICE  keys of the leader
  *   window_scores  DEVICE  out, float [B, H_kv, wkv_kw_max()] ; entries >= K_w,b are not written
  *   token_scores   DEVICE  out or NULL, float [B, H_kv, max(1, max_seqlen - alpha)] ; t_j of Eq. 2
- *   workspace      DEVICE  scratch of wkv_workspace_bytes() bytes.  Its first int32 is a status
- *                  word that the kernels only ever OR into (bit 0: a bounded wait inside a kernel
- *                  expired, results invalid): zero the workspace once after allocating it and read
- *                  the word whenever convenient.
+ *   workspace      DEVICE  scratch of wkv_workspace_bytes() bytes.  Zero it once after allocating
+ *                  it.  Its first int32 is a status word that the kernels only ever OR into
+ *                  (bit 0: a bounded wait inside a kernel expired, results invalid); the words
+ *                  behind it synchronise the blocks of a launch and reset themselves when the
+ *                  launch ends normally.  After a non-zero status zero the workspace again.
+ *                  One workspace serves one launch at a time.
  */
 int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader,
                       float *window_scores, float *token_scores,
