@@ -553,6 +553,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             Item im;
             make_item(u0 + item / cpu, item % cpu, 1, im);
             const int kw = num_windows(im.n, s.alpha, s.omega);
+            // read now, needed only by the block that selects: the load is long done by then
+            const int budget = a.window_idx ? (s.budgets ? __ldg(s.budgets + im.b) : s.budget) : 0;
             if (im.n_r <= 0 || im.n_tiles == 0) {
                 // a unit without review context still gets its (empty) selection, from its first item
                 if (a.window_idx && im.n_r <= 0 && im.chunk == 0) {
@@ -680,9 +682,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 }
                 __syncthreads();
                 if (flag_s) {
-                    const SeqInfo si = seq_info(s, im.b);
                     select_topk_block<kThreads>(topk_sm, a.window_scores + (size_t)im.unit * s.kw_max, kw,
-                                                num_selected(im.n, s.alpha, s.omega, si.budget), s.k_max,
+                                                num_selected(im.n, s.alpha, s.omega, budget), s.k_max,
                                                 a.window_idx + (size_t)im.unit * s.k_max, a.kept_len + im.unit,
                                                 im.n, s.alpha, s.omega);
                 }

@@ -64,12 +64,10 @@ __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total
 // All NT threads of the block call this.  `sc` are the unit's kw window scores (read through L2,
 // so scores written by other blocks of the same grid are seen once the caller has synchronised
 // with them), `out` receives k ascending indices followed by -1 up to k_max.
-// Thread t owns the windows [t*E, (t+1)*E), E = ceil(kw / NT).  With E <= kTopkRegs the keys are
-// read once and stay in registers through the radix passes and the compaction (one trip to L2
-// instead of five); longer lists are re-read.
-constexpr int kTopkRegs = 4;
-
-template <int NT, bool IN_REGS>
+// Thread t owns the windows [t*E, (t+1)*E), E = ceil(kw / NT).  With E <= REGS (4 or 8) the keys
+// are read once and stay in registers through the radix passes and the compaction (one trip to L2
+// instead of five); REGS = 0: longer lists are re-read.
+template <int NT, int REGS>
 __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, int kw, int k, int *out,
                                                  int *kept_len_out, int n, int alpha, int omega, int obs_rows)
 {
@@ -79,6 +77,8 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     static_assert(NT >= 256, "block size");
     const int E = (kw + NT - 1) / NT;
     const int w_lo = min(kw, (int)threadIdx.x * E), w_hi = min(kw, w_lo + E);
+    constexpr bool IN_REGS = REGS > 0;
+    constexpr int kTopkRegs = IN_REGS ? REGS : 1;
     unsigned keys[kTopkRegs];
     if (IN_REGS) {
 #pragma unroll
@@ -176,7 +176,7 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     }
     int eq_rank, pos;   // threshold keys before this thread; output position of its first selected window
     if (IN_REGS) {
-        // at most NT * kTopkRegs < 2^15 windows: both counts travel through one scan
+        // at most NT * 8 < 2^15 windows: both counts travel through one scan
         int total;
         const int both = topk_block_scan<NT>((n_eq << 16) | n_gt, sm.warp_sums, total);
         eq_rank = both >> 16;
@@ -225,10 +225,13 @@ __device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, 
         if (threadIdx.x == 0) *kept_len_out = obs_rows;
         return;
     }
-    if ((kw + NT - 1) / NT <= kTopkRegs)
-        select_topk_impl<NT, true>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+    const int per_thread = (kw + NT - 1) / NT;
+    if (per_thread <= 4)
+        select_topk_impl<NT, 4>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+    else if (per_thread <= 8)
+        select_topk_impl<NT, 8>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
     else
-        select_topk_impl<NT, false>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+        select_topk_impl<NT, 0>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
 }
 
 }  // namespace wkv
