@@ -111,6 +111,47 @@ def test_token_major_key_layout(impl):
         np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][layer]), ref["v_out"][layer])
 
 
+def test_more_work_items_than_blocks():
+    # 208 units of 300 keys: more (unit, chunk) items than SMs, so blocks take several items of
+    # different units (Q image reloaded, barrier phases carried across items)
+    w = small(batch=26, n_q_heads=16, n_kv_heads=8, head_dim=64, max_seqlen=300, l_obs=8, window=4,
+              budget_frac=0.25, n_planted=3, n_layers=1, gamma=1)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=IMPLS["tc"])
+    assert max_rel < 1e-4
+
+
+def test_long_window_list_is_reread_by_the_selection():
+    # 10,000 windows per unit: more than 8 per thread of the selecting block, which then streams
+    # the scores from L2 in every radix pass instead of holding them in registers
+    w = small(batch=1, n_q_heads=4, n_kv_heads=2, head_dim=64, max_seqlen=40008, l_obs=8, window=4,
+              budget_frac=0.1, n_planted=20, n_layers=1, gamma=1)
+    for impl in ("tc", "simt"):
+        grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=IMPLS[impl])
+        assert gpu["prob"].kw_max == 10000 and max_rel < 1e-4
+
+
+def test_one_workspace_serves_different_problems_in_turn():
+    # the synchronisation words in the workspace reset themselves at the end of every launch
+    cases = [small(), small(max_seqlen=2100, n_q_heads=8, n_kv_heads=1, l_obs=32), small(head_dim=64, window=4, l_obs=8)]
+    probs = [binding.Problem.from_workload(w) for w in cases]
+    work = torch.zeros(max(p.workspace_bytes for p in probs), dtype=torch.uint8, device="cuda")
+    for rep in range(2):
+        for w, prob in zip(cases, probs):
+            grp = wl.make_group(w, 0)
+            ref = oracle.select_leader(grp["q_obs"], grp["k_layers"][0], **pu.oracle_kwargs(w, grp))
+            q = binding.to_device(grp["q_obs"])
+            ks = [binding.to_device(x) for x in grp["k_layers"]]
+            vs = [binding.to_device(x) for x in grp["v_layers"]]
+            out = prob.alloc_outputs(len(ks), fill_byte=pu.FILL_BYTE)
+            binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
+                                       out["window_idx"], out["kept_len"], work, keep_capacity=out["keep_capacity"])
+            torch.cuda.synchronize()
+            assert binding.device_status(work) == 0
+            gpu = {"window_scores": out["window_scores"].cpu().numpy(), "window_idx": out["window_idx"].cpu().numpy(),
+                   "kept_len": out["kept_len"].cpu().numpy()}
+            pu.check_selection(w, grp, gpu, ref)
+
+
 def test_same_result_twice_and_across_entry_points():
     w = small()
     grp = wl.make_group(w, 0)
