@@ -547,6 +547,9 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
 
         grid_barrier(a.sync, gridDim.x, wave + 1, &abort_s);
         if (abort_s) break;
+        // behind the last barrier nobody polls the barrier word any more: sign off now, so that the
+        // round trip of this atomic is not on the way out of the kernel
+        if (wave + 1 == n_waves && threadIdx.x == 0) grid_barrier_leave(a.sync, gridDim.x);
 
         // ------------------------------------------------------------------ sweep 2 (+ selection)
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -705,7 +708,6 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             }
         }
         if (abort_s) atomicOr(a.status, kStatusWaitExpired);
-        else grid_barrier_leave(a.sync, gridDim.x);
     }
     tc_fence_before_sync();
     __syncthreads();
