@@ -1,5 +1,6 @@
 // Budgeted window selection (sentence after Eq. 4) for one unit by one thread block: the k-th
-// largest window score is found with a 3-pass radix select (11 + 11 + 10 bits) over an
+// largest window score is found with a radix select (11 bits per pass, only over the bits in which
+// the unit's keys differ, finished by direct ranking once few candidates are left) over an
 // order-preserving integer image of the fp32 scores, then the selected window indices are emitted
 // in ascending order with one block-wide prefix sum.  Equal scores at the threshold go to the
 // lower window index.  Integer arithmetic only after the key mapping, so the result is exact and
@@ -18,7 +19,11 @@ struct TopkSmem {
     unsigned prefix;
     int remaining;
     int last_selected;
+    unsigned kmin, kmax;        // smallest and largest key of the unit
+    int cand_total, n_cand;     // keys in the chosen bin; candidates collected for the direct finish
+    unsigned cand[64];
 };
+constexpr int kTopkDirect = 64;  // with at most this many candidates left, rank them directly
 
 // larger float <=> larger key; -0 and +0 map to the same key
 __device__ __forceinline__ unsigned topk_order_key(float f)
@@ -87,29 +92,91 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     auto key_at = [&](int e) -> unsigned { return IN_REGS ? keys[e] : topk_order_key(__ldcg(sc + w_lo + e)); };
 
     // ---- radix select: key of the k-th largest score --------------------------------
+    // Keys are taken relative to the smallest one, and only the bits in which the largest differs
+    // from it are resolved, 11 at a time from the top (window scores share sign and most of the
+    // exponent: typically one pass), until at most kTopkDirect candidates share the prefix; those
+    // are ranked against each other directly.
     if (threadIdx.x == 0) {
         sm.prefix = 0u;
         sm.remaining = k;
         sm.last_selected = 0;
+        sm.kmin = 0xffffffffu;
+        sm.kmax = 0u;
+        sm.cand_total = kw;
+        sm.n_cand = 0;
     }
     for (int x = threadIdx.x; x < kTopkBins; x += NT) sm.hist[x] = 0;
     __syncthreads();
+    {
+        unsigned lo = 0xffffffffu, hi = 0u;
+        if (IN_REGS) {
+#pragma unroll
+            for (int e = 0; e < kTopkRegs; ++e)
+                if (w_lo + e < w_hi) {
+                    lo = min(lo, keys[e]);
+                    hi = max(hi, keys[e]);
+                }
+        } else {
+            for (int e = 0; w_lo + e < w_hi; ++e) {
+                const unsigned key = key_at(e);
+                lo = min(lo, key);
+                hi = max(hi, key);
+            }
+        }
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        if ((threadIdx.x & 31) == 0) {
+            atomicMin(&sm.kmin, lo);
+            atomicMax(&sm.kmax, hi);
+        }
+    }
+    __syncthreads();
+    const unsigned kmin = sm.kmin;
+    const int bits = 32 - __clz(sm.kmax - kmin);     // 0 when all keys are equal
     unsigned mask = 0u;
+    int top = bits;                                   // bits [top, 32) of (key - kmin) are resolved
 #pragma unroll 1
-    for (int pass = 0; pass < 3; ++pass) {
-        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-        const unsigned digit_mask = pass == 2 ? 1023u : 2047u;
+    while (top > 0) {
         const unsigned prefix = sm.prefix;
         const int remaining = sm.remaining;
+        if (sm.cand_total <= kTopkDirect) {
+            // direct finish: collect the candidates, rank each against the others
+#pragma unroll
+            for (int e = 0; e < (IN_REGS ? kTopkRegs : E); ++e) {
+                if (IN_REGS && e >= E) break;
+                if (w_lo + e < w_hi) {
+                    const unsigned rk = key_at(e) - kmin;
+                    if ((rk & mask) == prefix) sm.cand[atomicAdd(&sm.n_cand, 1)] = rk;
+                }
+            }
+            __syncthreads();
+            const int n_cand = sm.n_cand;
+            if ((int)threadIdx.x < n_cand) {
+                const unsigned my = sm.cand[threadIdx.x];
+                int gt = 0, eq = 0;
+                for (int j = 0; j < n_cand; ++j) {
+                    const unsigned o = sm.cand[j];
+                    gt += o > my;
+                    eq += o == my;
+                }
+                if (gt < remaining && remaining <= gt + eq) {   // every thread that gets here writes the same values
+                    sm.prefix = my;
+                    sm.remaining = remaining - gt;
+                }
+            }
+            __syncthreads();
+            break;
+        }
+        const int low = top > 11 ? top - 11 : 0;
+        const unsigned digit_mask = (1u << (top - low)) - 1u;
 #pragma unroll
         for (int e = 0; e < (IN_REGS ? kTopkRegs : E); ++e) {
             if (IN_REGS && e >= E) break;   // uniform: E is the same for every thread
             unsigned bin = kTopkBins;       // not taking part in this pass
             if (w_lo + e < w_hi) {
-                const unsigned key = key_at(e);
-                if ((key & mask) == prefix) bin = (key >> shift) & digit_mask;
+                const unsigned rk = key_at(e) - kmin;
+                if ((rk & mask) == prefix) bin = (rk >> low) & digit_mask;
             }
-            // window scores share sign and exponent, so the keys of a warp often fall into one bin:
             // the lanes that share the bin of the first participating lane are counted by that lane
             const unsigned part = __ballot_sync(0xffffffffu, bin < kTopkBins);
             if (part) {
@@ -145,17 +212,19 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
             for (int i = kBinsPer - 1; i >= 0; --i) {
                 if (c[i] >= rem) {
                     bin = threadIdx.x * kBinsPer + i;
+                    sm.cand_total = c[i];
                     break;
                 }
                 rem -= c[i];
             }
-            sm.prefix = prefix | ((unsigned)bin << shift);
+            sm.prefix = prefix | ((unsigned)bin << low);
             sm.remaining = rem;   // after the last pass: how many keys equal to the threshold are taken
         }
-        mask |= digit_mask << shift;
+        mask |= digit_mask << low;
+        top = low;
         __syncthreads();
     }
-    const unsigned thr = sm.prefix;
+    const unsigned thr = sm.prefix + kmin;
     const int need_eq = sm.remaining;
 
     // ---- ordered compaction ----------------------------------------------------------
