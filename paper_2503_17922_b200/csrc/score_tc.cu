@@ -3,7 +3,8 @@
 //
 // The token score of Eq. 2, t_j = sum_i exp(s_ij) / Z_i, needs every row's softmax normaliser
 // Z_i (a reduction over all keys) before any column sum can be finished, so the keys are swept
-// twice, with a grid-wide barrier in between:
+// twice; a block starts normalising a unit's keys once all chunks of that unit have delivered their
+// sweep-1 statistics (a per-unit arrival count, no grid-wide barrier):
 //   sweep 1  D[rows, keys] = Q K^T per 128-key tile with the observation rows on the tensor-memory
 //            lanes: one thread owns one row and keeps its running (max, sum exp2) without any
 //            cross-thread traffic (Eq. 1's normaliser, causal mask on the tiles that touch the
@@ -22,7 +23,7 @@
 // contraction is the only tensor-core work; exponentials, sums and pooling are fp32 on the CUDA
 // cores in a fixed order, so results are bit-identical from run to run.
 //
-// Every wait is bounded (mbarriers and the grid barrier): on expiry the block sets bit 0 of the
+// Every wait is bounded (mbarriers and the wait for a unit's statistics): on expiry the block sets bit 0 of the
 // status word, drains its own TMA loads, frees its tensor memory and returns.
 #include "tc_common.cuh"
 #include "topk_block.cuh"
@@ -46,7 +47,7 @@ __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
 constexpr int kChunkCap = kTcMaxChunkTiles * kTile + kTcMaxWindow;   // token scores a block may hold
-constexpr int kSyncTickets = 16;                         // sync[0..1] grid barrier, tickets from sync[16]
+constexpr int kSyncTickets = 16;                         // per unit u: sync[16 + 2u] ticket, sync[17 + 2u] sweep-1 arrivals
 
 struct TcArgs {
     KShape s;
@@ -105,47 +106,45 @@ __device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
     if (lane == 0) mbar_arrive(bar);
 }
 
-// Grid-wide barrier of a cooperative launch (all blocks resident).  sync[0] counts arrivals and only
-// grows during a launch: the barrier number `phase` is passed once n_blocks * phase blocks have
-// arrived (one atomic and one polled word per barrier).  sync[1] counts the blocks that have left
-// the kernel; the last one clears both words for the next launch.  Bounded: a block that waits
-// longer than two seconds gives up, sets its abort flag and the caller tears the block down.
+// Hand-over between the sweeps, per unit (all blocks are resident: cooperative launch).  A block that
+// has written the sweep-1 statistics of one chunk adds one to the unit's arrival word; a block about
+// to normalise keys of the unit waits until all of the unit's chunks have arrived.  No block waits
+// before it has finished all its sweep-1 work, so every wait ends.  The block that takes the unit's
+// last ticket in sweep 2 (every waiter of the unit is past its wait by then) clears both words for
+// the next launch.  Bounded: a warp that waits longer than two seconds gives up and sets the
+// block's abort flag.
 __device__ __forceinline__ int ld_acquire_gpu(const int *p)
 {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void grid_barrier(int *sync, int n_blocks, int phase, volatile int *abort_flag)
+__device__ __forceinline__ void red_release_gpu_add(int *p, int v)
 {
-    __syncthreads();
-    if (threadIdx.x == 0 && !*abort_flag) {
-        // the fence of thread 0 is cumulative: it also publishes what the other threads of the block
-        // wrote before the block barrier above
-        __threadfence();
-        atomicAdd(sync, 1);
-        const int target = n_blocks * phase;
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool warp_wait_arrivals(const int *word, int target, volatile int *abort_flag, int lane)
+{
+    int ok = 1;
+    if (lane == 0) {
         unsigned long long t0 = 0;
-        for (uint32_t spin = 1; ld_acquire_gpu(sync) < target; ++spin) {
-            if ((spin & 1023u) == 0u) {
+        for (uint32_t spin = 1; ld_acquire_gpu(word) < target; ++spin) {
+            if (*abort_flag) {
+                ok = 0;
+                break;
+            }
+            if ((spin & 255u) == 0u) {
                 const unsigned long long now = global_timer_ns();
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > 2 * kWaitLimitNs) {
                     *abort_flag = 1;
+                    ok = 0;
                     break;
                 }
             }
         }
-        __threadfence();
     }
-    __syncthreads();
-}
-__device__ __forceinline__ void grid_barrier_leave(int *sync, int n_blocks)
-{
-    if (atomicAdd(sync + 1, 1) == n_blocks - 1) {
-        atomicExch(sync, 0);
-        atomicExch(sync + 1, 0);
-    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // geometry of one work item
@@ -543,13 +542,10 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 out[r] = res;
             }
             __syncthreads();   // `part` is rewritten by the next item
+            // release: cumulative over what the block wrote before the barrier above
+            if (threadIdx.x == 0) red_release_gpu_add(a.sync + kSyncTickets + 2 * im.unit + 1, 1);
         }
-
-        grid_barrier(a.sync, gridDim.x, wave + 1, &abort_s);
         if (abort_s) break;
-        // behind the last barrier nobody polls the barrier word any more: sign off now, so that the
-        // round trip of this atomic is not on the way out of the kernel
-        if (wave + 1 == n_waves && threadIdx.x == 0) grid_barrier_leave(a.sync, gridDim.x);
 
         // ------------------------------------------------------------------ sweep 2 (+ selection)
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -586,11 +582,14 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 constexpr int kMergers = kComputeThreads / q_rows;
                 float2 *merged = &part[0][0][0];
                 const int tl = threadIdx.x - 64;
-                if (tl < kMergers * q_rows) {
+                const int len1 = tc_chunk_len(im.n, cpu, 1);
+                const int used1 = (im.n + len1 - 1) / len1;   // chunks of the unit that hold keys in sweep 1
+                const bool arrived =
+                    warp_wait_arrivals(a.sync + kSyncTickets + 2 * im.unit + 1, used1, &abort_s, lane);
+                if (tl < kMergers * q_rows && arrived) {
                     const int r = tl % q_rows, mp = tl / q_rows;
                     float M = -INFINITY, sum = 0.f;
-                    const int len1 = tc_chunk_len(im.n, cpu, 1);
-                    const int used = r < s.R ? (im.n + len1 - 1) / len1 : 0;
+                    const int used = r < s.R ? used1 : 0;
                     const float2 *st = a.stats + (size_t)im.unit * a.n_stat_chunks * a.r_pad + r;
                     for (int c0 = mp; c0 < used || c0 == mp; c0 += 8 * kMergers) {
                         float2 p[8];
@@ -668,17 +667,27 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                     }
                 }
             }
-            if (a.window_idx) {
+            const int len2 = tc_chunk_len(im.n_r, cpu, s.omega);
+            const int used2 = (im.n_r + len2 - 1) / len2;   // chunks of the unit that hold keys in sweep 2
+            if (!a.window_idx) {
+                // nothing to publish: the ticket only finds the block that clears the unit's words
+                if (threadIdx.x == 0) {
+                    int *ticket = a.sync + kSyncTickets + 2 * im.unit;
+                    if (atomicAdd(ticket, 1) == used2 - 1) {
+                        atomicExch(ticket, 0);
+                        atomicExch(ticket + 1, 0);
+                    }
+                }
+            } else {
                 // the block that completes the unit's last windows selects for the unit
-                const int len2 = tc_chunk_len(im.n_r, cpu, s.omega);
-                const int used2 = (im.n_r + len2 - 1) / len2;
                 __syncthreads();
                 if (threadIdx.x == 0) {
                     __threadfence();   // cumulative: publishes the window scores the whole block wrote
-                    int *ticket = a.sync + kSyncTickets + im.unit;
+                    int *ticket = a.sync + kSyncTickets + 2 * im.unit;
                     const int last = atomicAdd(ticket, 1) == used2 - 1;
                     if (last) {
                         atomicExch(ticket, 0);
+                        atomicExch(ticket + 1, 0);
                         __threadfence();
                     }
                     flag_s = last;
@@ -884,7 +893,7 @@ int launch_score_tc(const KShape &ks, const void *q, const void *k, float *windo
         }
     }
     // persistent blocks, one per SM at most; every block of a cooperative launch is resident, which
-    // the grid barrier between the sweeps relies on
+    // the hand-over of the statistics between the sweeps relies on
     int grid = plan.units_per_wave * plan.chunks_per_unit;
     if (grid > di.sm_count) grid = di.sm_count;
     const __nv_bfloat16 *qp = static_cast<const __nv_bfloat16 *>(q);

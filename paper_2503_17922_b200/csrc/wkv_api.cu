@@ -39,7 +39,7 @@ Workspace plan_workspace(const KShape &ks)
     w.status_off = off;
     off = 64;
     w.sync_off = off;
-    off = align_up(off + (16 + units) * sizeof(int), 256);
+    off = align_up(off + (16 + 2 * (size_t)units) * sizeof(int), 256);
     w.stats_off = off;
     off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
     w.lse_off = off;

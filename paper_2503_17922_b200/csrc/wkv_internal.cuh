@@ -64,7 +64,7 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
     size_t status_off;   // int: device status word, only ever OR-ed by the kernels (0 = no error)
-    size_t sync_off;     // int [16 + units]: grid-barrier count and generation, per-unit tickets (self-resetting)
+    size_t sync_off;     // int [16 + 2 * units]: per unit a ticket and a count of sweep-1 arrivals (self-resetting)
     size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
     size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
     size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none
