@@ -41,6 +41,7 @@ namespace {
 using namespace tc;
 
 constexpr int kStages = 4;
+constexpr int kEarlyTiles = 2;                           // key tiles requested ahead of the Q image at the start of an item
 constexpr int kMaxGroups = 4;
 __host__ __device__ constexpr int groups_for(int mb) { return mb == 1 ? 4 : 2; }
 __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for(mb) * 128; }
@@ -153,7 +154,17 @@ struct Item {
     int n, n_r;
     long long off;
     int j_begin, j_end, n_tiles;
+    int reuse;   // sweep 2: the stage ring still holds the item's last tiles from sweep 1
 };
+// Tile taken at step u of an item.  Sweep 1 and a sweep 2 that has to load everything go through the
+// tiles in ascending order.  A block that scores the item it has just taken statistics of still holds
+// that item's last kStages tiles in the ring, in ring order: it scores those first, without
+// loading them again, and then walks down through the rest.
+__device__ __forceinline__ int tile_at(const Item &im, int u)
+{
+    if (!im.reuse) return u;
+    return u < kStages ? im.n_tiles - kStages + u : im.n_tiles - 1 - u;
+}
 
 // ---------------------------------------------------------------------------------------------
 // per-element work of the two sweeps
@@ -291,6 +302,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     int q_unit_loaded = -1;
     uint32_t it = 0;            // key tiles this block has pushed through the pipeline so far
     uint32_t p_issued = 0;      // producer thread only: tiles whose loads have been issued
+    int s1_unit = -1, s1_chunk = -1, s1_tiles = 0;   // the sweep-1 item whose last tiles the ring holds ...
+    uint32_t s1_it = 0;                              // ... as long as `it` still has this value
 
     auto make_item = [&](int unit, int chunk, int review_only, Item &im) {
         im.unit = unit;
@@ -311,6 +324,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.j_begin = chunk * len;
         im.j_end = min(n_keys, im.j_begin + len);
         im.n_tiles = im.j_end > im.j_begin ? (im.j_end - im.j_begin + kTile - 1) / kTile : 0;
+        im.reuse = 0;
     };
 
     // Called by every warp except the producer; ends with a barrier among those warps.  Four loads
@@ -357,15 +371,21 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     };
 
     // producer: the item's key tiles into the stage ring (the block-wide tile counter `it` keeps the phases)
-    auto produce = [&](const Item &im) {
+    auto produce = [&](const Item &im, int t_begin, int t_end) {
         const int tok0 = (int)im.off + im.j_begin;
         const int bcoord = s.cu ? 0 : im.b;
-        for (int t = 0; t < im.n_tiles; ++t) {
+        for (int t = t_begin; t < t_end; ++t) {
             const uint32_t g = it + t;
             const int st = g % kStages;
+            if (im.reuse && t < kStages) {
+                // the stage holds this tile already: complete the phase without a load
+                mbar_arrive(&bar.full[st]);
+                ++p_issued;
+                continue;
+            }
             if (g >= kStages && !mbar_wait(&bar.empty[st], ((g / kStages) - 1) & 1, &abort_s)) return;
             mbar_arrive_expect_tx(&bar.full[st], (uint32_t)stage_bytes);
-            const int tok = tok0 + t * kTile;
+            const int tok = tok0 + tile_at(im, t) * kTile;
             const int c1 = a.slot_tok == 1 ? tok : (a.slot_h == 1 ? im.h : bcoord);
             const int c2 = a.slot_tok == 2 ? tok : (a.slot_h == 2 ? im.h : bcoord);
             const int c3 = a.slot_tok == 3 ? tok : (a.slot_h == 3 ? im.h : bcoord);
@@ -482,7 +502,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 score_accumulate<16>(vt, neg_lse2 + n32 * 32, c, a0, a1, a2, a3);
             }
             const float tj = (a0 + a1) + (a2 + a3);
-            const int j = im.j_begin + t * kTile + L;
+            const int j = im.j_begin + tile_at(im, t) * kTile + L;
             if (j < im.j_end) {
                 t_chunk[j - im.j_begin] = tj;
                 if (a.token_scores) a.token_scores[(size_t)im.unit * s.nr_max + j] = tj;
@@ -506,8 +526,12 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 continue;
             }
             if (warp == 0) {
+                // the first tiles leave before the loads of the Q image (they land while those are
+                // being issued); the rest of the ring's burst follows once the Q loads are on their way
+                const int early = min(kEarlyTiles, im.n_tiles);
+                if (lane == 0) produce(im, 0, early);
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
-                if (lane == 0) produce(im);
+                if (lane == 0) produce(im, early, im.n_tiles);
             } else {
                 load_q_image(im, true);
                 if (warp == 1) {
@@ -518,6 +542,10 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             }
             q_unit_loaded = im.unit;
             it += im.n_tiles;
+            s1_unit = im.unit;
+            s1_chunk = im.chunk;
+            s1_tiles = im.n_tiles;
+            s1_it = it;
             tc_fence_before_sync();
             __syncthreads();
             tc_fence_after_sync();
@@ -564,9 +592,14 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 }
                 continue;
             }
+            const int len1 = tc_chunk_len(im.n, cpu, 1);
+            im.reuse = im.unit == s1_unit && im.chunk == s1_chunk && it == s1_it && im.n_tiles == s1_tiles &&
+                       im.n_tiles >= kStages && im.chunk * len1 == im.j_begin;
             if (warp == 0) {
+                const int held = im.reuse ? kStages : 0;
+                if (lane == 0) produce(im, 0, held);
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
-                if (lane == 0) produce(im);
+                if (lane == 0) produce(im, held, im.n_tiles);
             } else {
                 load_q_image(im, false);
                 if (warp == 1) {
@@ -582,7 +615,6 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 constexpr int kMergers = kComputeThreads / q_rows;
                 float2 *merged = &part[0][0][0];
                 const int tl = threadIdx.x - 64;
-                const int len1 = tc_chunk_len(im.n, cpu, 1);
                 const int used1 = (im.n + len1 - 1) / len1;   // chunks of the unit that hold keys in sweep 1
                 const bool arrived =
                     warp_wait_arrivals(a.sync + kSyncTickets + 2 * im.unit + 1, used1, &abort_s, lane);
