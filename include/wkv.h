@@ -205,6 +205,30 @@ int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_l
                        void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Scoring and the whole group for callers that already hold Eq. 1's normalisers.  The prefill
+ * attention of the leader layer computes, for every query row, the log-sum-exp of its causal
+ * softmax; handing in the values of the observation rows removes the pass over the keys that
+ * otherwise recomputes them (the keys are then read once and never re-read).
+ *   lse_obs   DEVICE float [B, H_q, alpha], contiguous: natural log of
+ *             sum_{j <= position(i)} exp(q_i . k_j / sqrt(d)) for observation row i of query
+ *             head h (row i of head h at (b * H_q + h) * alpha + i), over ALL keys the row may
+ *             attend to, observation-window keys included (Eq. 1's denominator).
+ * Everything else as in wkv_score_windows / wkv_compress_group.  Values that are not the
+ * normalisers of q_obs and k_leader give scores that are wrong by the corresponding factor per
+ * row; nothing checks them.  NULL lse_obs is an error (WKV_ERR_NULL).
+ */
+int wkv_score_windows_lse(const wkv_shape *s, const void *q_obs, const void *k_leader,
+                          const float *lse_obs, float *window_scores, float *token_scores,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+int wkv_compress_group_lse(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
+                           const float *lse_obs,
+                           const void *const *k_layers, const void *const *v_layers,
+                           void *const *k_out_layers, void *const *v_out_layers,
+                           float *window_scores, int32_t *window_idx, int32_t *kept_len,
+                           const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The same group with every tensor in HOST memory (pinned memory recommended): the
  * inputs are copied to caller-provided DEVICE staging buffers, the group is
  * compressed there, and indices, kept lengths and the compact caches are copied

@@ -24,7 +24,7 @@ WKV_MAX_GROUP_LAYERS = 32
 EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
-    "wkv_compress_group", "wkv_compress_group_host", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
 
@@ -100,6 +100,10 @@ def lib() -> ctypes.CDLL:
     L.wkv_gather_kv.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
     L.wkv_compress_group.restype = ctypes.c_int
     L.wkv_compress_group.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.wkv_score_windows_lse.restype = ctypes.c_int
+    L.wkv_score_windows_lse.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.wkv_compress_group_lse.restype = ctypes.c_int
+    L.wkv_compress_group_lse.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     L.wkv_compress_group_host.restype = ctypes.c_int
     L.wkv_compress_group_host.argtypes = [sp, i32, vp, sz, vp, vp, sz, vp, vp, sz, vp, vp,
                                           vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
@@ -277,6 +281,33 @@ def wkv_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_out_la
                                     workspace.numel(), _stream(stream)), "wkv_compress_group")
 
 
+def wkv_score_windows_lse(prob: Problem, q_obs, k_leader, lse_obs, window_scores, token_scores, workspace,
+                          stream=None) -> None:
+    """Scoring with the observation rows' softmax normalisers (natural-log LSE, float [B, H_q, alpha])
+    supplied by the caller, e.g. from the leader layer's prefill attention."""
+    _check(lib().wkv_score_windows_lse(ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader), _ptr(lse_obs),
+                                       _ptr(window_scores), _ptr(token_scores), _ptr(workspace), workspace.numel(),
+                                       _stream(stream)), "wkv_score_windows_lse")
+
+
+def _group_lse_args(prob, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers, window_scores,
+                    window_idx, kept_len, workspace, cu_seqlens_out, keep_capacity, stream):
+    arrs = (_ptr_array(k_layers), _ptr_array(v_layers), _ptr_array(k_out_layers), _ptr_array(v_out_layers))
+    args = (ctypes.byref(prob.shape), len(k_layers), _ptr(q_obs_leader), _ptr(lse_obs), arrs[0], arrs[1], arrs[2],
+            arrs[3], _ptr(window_scores), _ptr(window_idx), _ptr(kept_len), _ptr(cu_seqlens_out), keep_capacity,
+            _ptr(workspace), workspace.numel(), _stream(stream))
+    return args, arrs
+
+
+def wkv_compress_group_lse(prob: Problem, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                           window_scores, window_idx, kept_len, workspace, cu_seqlens_out=None,
+                           keep_capacity: int = 0, stream=None) -> None:
+    args, _keep = _group_lse_args(prob, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                                  window_scores, window_idx, kept_len, workspace, cu_seqlens_out, keep_capacity,
+                                  stream)
+    _check(lib().wkv_compress_group_lse(*args), "wkv_compress_group_lse")
+
+
 class PreparedCall:
     """A C-ABI call with its arguments marshalled once (pointer tables, shape, stream): `run()` is a
     single foreign call, so that a loop over many groups is not bound by Python."""
@@ -300,6 +331,17 @@ def prepare_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_ou
     return PreparedCall(lib().wkv_compress_group, "wkv_compress_group", args,
                         (prob, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers, window_scores,
                          window_idx, kept_len, workspace, cu_seqlens_out, arrs))
+
+
+def prepare_compress_group_lse(prob: Problem, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers,
+                               v_out_layers, window_scores, window_idx, kept_len, workspace, cu_seqlens_out=None,
+                               keep_capacity: int = 0, stream=None) -> PreparedCall:
+    args, arrs = _group_lse_args(prob, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                                 window_scores, window_idx, kept_len, workspace, cu_seqlens_out, keep_capacity,
+                                 stream)
+    return PreparedCall(lib().wkv_compress_group_lse, "wkv_compress_group_lse", args,
+                        (prob, arrs, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                         window_scores, window_idx, kept_len, workspace, cu_seqlens_out))
 
 
 def prepare_score_windows(prob: Problem, q_obs, k_leader, window_scores, token_scores, workspace,

@@ -179,8 +179,9 @@ score_stats_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k, flo
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 score_pool_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k,
-                const float2 *__restrict__ stats, float *__restrict__ window_scores,
-                float *__restrict__ token_scores, int n_chunks, int r_pad, int chunk_keys)
+                const float2 *__restrict__ stats, const float *__restrict__ lse_obs,
+                float *__restrict__ window_scores, float *__restrict__ token_scores, int n_chunks, int r_pad,
+                int chunk_keys)
 {
     extern __shared__ __align__(16) float smem[];
     float *qs = smem;                          // [d][r_pad]
@@ -201,7 +202,14 @@ score_pool_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k,
     load_q_transposed(s, q_unit, qs, r_pad);
 
     // combine the partial statistics of every chunk: lse2 = log2 of the row normaliser
+    // (or, when the caller supplies the natural log of the normalisers, that value in base 2)
     for (int r = threadIdx.x; r < r_pad; r += kThreads) {
+        if (lse_obs) {
+            const int g = r / s.alpha, i = r - g * s.alpha;
+            lse2[r] = r < s.R ? lse_obs[((size_t)b * s.hq + (size_t)h * s.G + g) * s.alpha + i] * 1.4426950408889634f
+                              : INFINITY;
+            continue;
+        }
         const float2 *st = stats + (size_t)unit * n_chunks * r_pad + r;
         float M = -INFINITY;
         for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, st[(size_t)c * r_pad].x);
@@ -266,7 +274,7 @@ static int simt_chunk_keys(const KShape &ks)
 
 cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const void *k,
                               float *window_scores, float *token_scores,
-                              void *workspace, const Workspace &ws, cudaStream_t stream)
+                              void *workspace, const Workspace &ws, cudaStream_t stream, const float *lse_obs)
 {
     const int units = ks.batch * ks.hkv;
     const int r_pad = ws.r_pad;
@@ -288,10 +296,11 @@ cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const 
         err = cudaFuncSetAttribute(score_pool_simt<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
                                    (int)smem2);                                                     \
         if (err != cudaSuccess) return err;                                                         \
-        score_stats_simt<T><<<g1, kThreads, smem1, stream>>>(ks, (const T *)q, (const T *)k, stats, \
-                                                             ws.n_stat_chunks, r_pad);              \
+        if (!lse_obs)                                                                               \
+            score_stats_simt<T><<<g1, kThreads, smem1, stream>>>(ks, (const T *)q, (const T *)k, stats, \
+                                                                 ws.n_stat_chunks, r_pad);          \
         score_pool_simt<T><<<g2, kThreads, smem2, stream>>>(ks, (const T *)q, (const T *)k, stats,  \
-                                                            window_scores, token_scores,            \
+                                                            lse_obs, window_scores, token_scores,   \
                                                             ws.n_stat_chunks, r_pad, chunk_keys);   \
     } while (0)
     if (dtype == WKV_F32)
@@ -299,7 +308,7 @@ cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const 
     else
         WKV_LAUNCH_SIMT(__nv_bfloat16);
 #undef WKV_LAUNCH_SIMT
-    count_launches(2);
+    count_launches(lse_obs ? 1 : 2);
     return cudaGetLastError();
 }
 

@@ -55,6 +55,7 @@ struct TcArgs {
     float2 *stats;          // [units][n_stat_chunks][r_pad]
     float *window_scores;
     float *token_scores;
+    const float *lse_obs;   // [B, H_q, alpha] natural log of Eq. 1's normalisers from the caller, or null
     int *window_idx;        // fused selection when non-null
     int *kept_len;
     int *status;
@@ -517,7 +518,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         const int n_items = nu * cpu;
 
         // ------------------------------------------------------------------ sweep 1
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        // (not needed when the caller supplies the normalisers: sweep 2 then reads the keys from HBM)
+        for (int item = blockIdx.x; item < n_items && !a.lse_obs; item += gridDim.x) {
             Item im;
             make_item(u0 + item / cpu, item % cpu, 0, im);
             float2 *out = a.stats + ((size_t)im.unit * a.n_stat_chunks + im.chunk) * a.r_pad;
@@ -615,6 +617,21 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 constexpr int kMergers = kComputeThreads / q_rows;
                 float2 *merged = &part[0][0][0];
                 const int tl = threadIdx.x - 64;
+                if (a.lse_obs) {
+                    // the caller's normalisers, to base 2; row r = (query head g of the group, position i)
+                    if (tl < 256) {
+                        float v = -INFINITY;
+                        if (tl < s.R) {
+                            const int g = tl / s.alpha, i = tl - g * s.alpha;
+                            v = -1.4426950408889634f *
+                                __ldg(a.lse_obs + ((size_t)im.b * s.hq + (size_t)im.h * s.G + g) * s.alpha + i);
+                        }
+                        neg_lse2[tl] = v;
+                    }
+                    go_producer();
+                    asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
+                    compute_scores(im);
+                } else {
                 const int used1 = (im.n + len1 - 1) / len1;   // chunks of the unit that hold keys in sweep 1
                 const bool arrived =
                     warp_wait_arrivals(a.sync + kSyncTickets + 2 * im.unit + 1, used1, &abort_s, lane);
@@ -666,6 +683,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 }
                 asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
                 compute_scores(im);
+                }
                 }
             }
             q_unit_loaded = im.unit;
@@ -870,7 +888,8 @@ bool score_tc_supported(const KShape &ks, int dtype)
 }
 
 int launch_score_tc(const KShape &ks, const void *q, const void *k, float *window_scores, float *token_scores,
-                    int *window_idx, int *kept_len, void *workspace, const Workspace &ws, cudaStream_t stream)
+                    int *window_idx, int *kept_len, void *workspace, const Workspace &ws, cudaStream_t stream,
+                    const float *lse_obs)
 {
     alignas(64) CUtensorMap tmap;
     int slot[3] = {1, 2, 3};
@@ -881,6 +900,7 @@ int launch_score_tc(const KShape &ks, const void *q, const void *k, float *windo
     a.s = ks;
     a.stats = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + ws.stats_off);
     a.window_scores = window_scores;
+    a.lse_obs = lse_obs;
     a.token_scores = token_scores;
     a.window_idx = window_idx;
     a.kept_len = kept_len;

@@ -211,7 +211,7 @@ static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace
 
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
              float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
-             cudaStream_t stream)
+             cudaStream_t stream, const float *lse_obs)
 {
     if (!aligned16(q) || !aligned16(k)) {
         set_error_detail("q_obs / k_leader not 16-byte aligned");
@@ -221,12 +221,14 @@ int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const vo
     int st = pick_score_impl(s, ks, ws, use_tc);
     if (st != WKV_OK) return st;
     if (use_tc) {
-        st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream);
+        st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream,
+                             lse_obs);
         // a key layout that no tensor map can describe is served by the CUDA-core kernels
         if (st != WKV_ERR_UNSUPPORTED || s->score_impl == WKV_SCORE_TCGEN05) return st;
         if (score_simt_smem_bytes(ks, ws.r_pad) > 227u * 1024u) return st;
     }
-    st = check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream),
+    st = check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream,
+                                      lse_obs),
                     "score kernels");
     if (st == WKV_OK && window_idx)
         st = check_cuda(launch_topk(ks, window_scores, window_idx, kept_len, stream), "selection kernel");
@@ -348,8 +350,9 @@ size_t wkv_workspace_bytes(const wkv_shape *s)
     return plan_workspace(ks).total;
 }
 
-int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader, float *window_scores,
-                      float *token_scores, void *workspace, size_t workspace_bytes, void *cuda_stream)
+static int score_windows_entry(const wkv_shape *s, const void *q_obs, const void *k_leader, const float *lse_obs,
+                               float *window_scores, float *token_scores, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream)
 {
     KShape ks;
     int st = resolve(s, ks);
@@ -362,7 +365,26 @@ int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leade
     st = check_workspace(ws, workspace, workspace_bytes);
     if (st != WKV_OK) return st;
     return do_score(s, ks, ws, q_obs, k_leader, window_scores, token_scores, nullptr, nullptr, workspace,
-                    static_cast<cudaStream_t>(cuda_stream));
+                    static_cast<cudaStream_t>(cuda_stream), lse_obs);
+}
+
+int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leader, float *window_scores,
+                      float *token_scores, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return score_windows_entry(s, q_obs, k_leader, nullptr, window_scores, token_scores, workspace, workspace_bytes,
+                               cuda_stream);
+}
+
+int wkv_score_windows_lse(const wkv_shape *s, const void *q_obs, const void *k_leader, const float *lse_obs,
+                          float *window_scores, float *token_scores, void *workspace, size_t workspace_bytes,
+                          void *cuda_stream)
+{
+    if (!lse_obs) {
+        set_error_detail("lse_obs is NULL");
+        return WKV_ERR_NULL;
+    }
+    return score_windows_entry(s, q_obs, k_leader, lse_obs, window_scores, token_scores, workspace, workspace_bytes,
+                               cuda_stream);
 }
 
 int wkv_select_topk_windows(const wkv_shape *s, const float *window_scores, int32_t *window_idx,
@@ -404,11 +426,11 @@ int wkv_gather_kv(const wkv_shape *s, int32_t n_layers, const void *const *k_lay
                       "gather kernel");
 }
 
-int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
-                       const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
-                       void *const *v_out_layers, float *window_scores, int32_t *window_idx,
-                       int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
-                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+static int compress_group_entry(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader, const float *lse_obs,
+                                const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
+                                void *const *v_out_layers, float *window_scores, int32_t *window_idx,
+                                int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     KShape ks;
     int st = resolve(s, ks);
@@ -431,11 +453,38 @@ int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_l
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float *scores = window_scores ? window_scores
                                   : reinterpret_cast<float *>(static_cast<char *>(workspace) + ws.scores_off);
-    st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, window_idx, kept_len, workspace, stream);
+    st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, window_idx, kept_len, workspace, stream,
+                  lse_obs);
     if (st != WKV_OK) return st;
     return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
                                     keep_capacity, stream),
                       "gather kernel");
+}
+
+int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
+                       const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
+                       void *const *v_out_layers, float *window_scores, int32_t *window_idx,
+                       int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return compress_group_entry(s, n_layers, q_obs_leader, nullptr, k_layers, v_layers, k_out_layers, v_out_layers,
+                                window_scores, window_idx, kept_len, cu_seqlens_out, keep_capacity, workspace,
+                                workspace_bytes, cuda_stream);
+}
+
+int wkv_compress_group_lse(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader, const float *lse_obs,
+                           const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
+                           void *const *v_out_layers, float *window_scores, int32_t *window_idx,
+                           int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!lse_obs) {
+        set_error_detail("lse_obs is NULL");
+        return WKV_ERR_NULL;
+    }
+    return compress_group_entry(s, n_layers, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                                window_scores, window_idx, kept_len, cu_seqlens_out, keep_capacity, workspace,
+                                workspace_bytes, cuda_stream);
 }
 
 int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers, const void *q_obs_host, size_t q_bytes,

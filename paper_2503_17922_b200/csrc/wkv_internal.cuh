@@ -124,12 +124,15 @@ Workspace plan_workspace(const KShape &ks);
 // Launchers (each returns a cudaError_t from the launch).
 cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const void *k,
                               float *window_scores, float *token_scores,
-                              void *workspace, const Workspace &ws, cudaStream_t stream);
+                              void *workspace, const Workspace &ws, cudaStream_t stream,
+                              const float *lse_obs = nullptr);
 bool score_tc_supported(const KShape &ks, int dtype);
-// window_idx / kept_len non-null: the selection is fused into the same launch
+// window_idx / kept_len non-null: the selection is fused into the same launch.
+// lse_obs non-null: float [B, H_q, alpha], natural log of Eq. 1's normaliser of every observation
+// row, supplied by the caller; the statistics sweep is then skipped.
 int launch_score_tc(const KShape &ks, const void *q, const void *k,
                     float *window_scores, float *token_scores, int *window_idx, int *kept_len,
-                    void *workspace, const Workspace &ws, cudaStream_t stream);
+                    void *workspace, const Workspace &ws, cudaStream_t stream, const float *lse_obs = nullptr);
 cudaError_t launch_topk(const KShape &ks, const float *window_scores, int *window_idx, int *kept_len,
                         cudaStream_t stream);
 
@@ -176,7 +179,7 @@ int check_cuda(cudaError_t e, const char *what);         // cudaError_t -> wkv_s
 // scoring; with window_idx / kept_len non-null also the selection (one launch on the tensor-core path)
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
              float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
-             cudaStream_t stream);
+             cudaStream_t stream, const float *lse_obs = nullptr);
 
 void count_launches(int n);
 void set_error_detail(const char *fmt, ...);

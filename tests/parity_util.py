@@ -33,9 +33,36 @@ def fill_pattern(dtype: str) -> int:
     return 0xA5A5A5A5 if dtype == "f32" else 0xA5A5
 
 
-def run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_AUTO, staged=False, want_tokens=False):
+def lse_obs_reference(w, grp) -> np.ndarray:
+    """Eq. 1's normalisers as a prefill attention would hand them over: natural log of the sum of
+    exp(q_i . k_j / sqrt(d)) over the keys j <= position(i), for every observation row, float32
+    [B, H_q, alpha].  Plain numpy in float64, written out from the definition."""
+    q = wl.to_f32(grp["q_obs"]).astype(np.float64)          # [B, H_q, alpha, d]
+    k = wl.to_f32(grp["k_layers"][0]).astype(np.float64)
+    G = w.n_q_heads // w.n_kv_heads
+    out = np.zeros((w.batch, w.n_q_heads, w.l_obs), dtype=np.float32)
+    for b in range(w.batch):
+        n = int(grp["seqlens"][b])
+        if n <= w.l_obs:
+            continue                                         # nothing is scored for such a sequence
+        if grp["cu_seqlens"] is not None:
+            lo = int(grp["cu_seqlens"][b])
+            kb = k[lo:lo + n].transpose(1, 0, 2)             # packed [T, H_kv, d] -> [H_kv, n, d]
+        else:
+            kb = k[b, :, :n]
+        for hq in range(w.n_q_heads):
+            logits = q[b, hq] @ kb[hq // G].T / np.sqrt(w.head_dim)      # [alpha, n]
+            for i in range(w.l_obs):
+                row = logits[i, :n - w.l_obs + i + 1]
+                m = row.max()
+                out[b, hq, i] = m + np.log(np.exp(row - m).sum())
+    return out
+
+
+def run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_AUTO, staged=False, want_tokens=False, lse_obs=None):
     """Runs the whole group on the GPU. `staged` uses the three stage entry points
-    instead of wkv_compress_group.  Returns host copies of every output."""
+    instead of wkv_compress_group; `lse_obs` (host float32 [B, H_q, alpha]) the entry points
+    that take the normalisers from the caller.  Returns host copies of every output."""
     prob = binding.Problem.from_workload(w, score_impl=score_impl)
     q = binding.to_device(grp["q_obs"])
     ks = [binding.to_device(x) for x in grp["k_layers"]]
@@ -43,16 +70,24 @@ def run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_AUTO, staged=False, want_
     out = prob.alloc_outputs(len(ks), fill_byte=FILL_BYTE)
     work = prob.alloc_workspace()
     tok = None
+    lse = None if lse_obs is None else torch.from_numpy(np.ascontiguousarray(lse_obs)).cuda()
     if staged:
         if want_tokens:
             tok = torch.full((w.batch, w.n_kv_heads, prob.nr_max), float("nan"), dtype=torch.float32, device="cuda")
-        binding.wkv_score_windows(prob, q, ks[0], out["window_scores"], tok, work)
+        if lse is None:
+            binding.wkv_score_windows(prob, q, ks[0], out["window_scores"], tok, work)
+        else:
+            binding.wkv_score_windows_lse(prob, q, ks[0], lse, out["window_scores"], tok, work)
         binding.wkv_select_topk_windows(prob, out["window_scores"], out["window_idx"], out["kept_len"])
         binding.wkv_gather_kv(prob, ks, vs, out["window_idx"], out["k_out"], out["v_out"],
                               keep_capacity=out["keep_capacity"])
-    else:
+    elif lse is None:
         binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
                                    out["window_idx"], out["kept_len"], work, keep_capacity=out["keep_capacity"])
+    else:
+        binding.wkv_compress_group_lse(prob, q, lse, ks, vs, out["k_out"], out["v_out"], out["window_scores"],
+                                       out["window_idx"], out["kept_len"], work,
+                                       keep_capacity=out["keep_capacity"])
     torch.cuda.synchronize()
     assert binding.device_status(work) == 0, "a kernel reported an expired wait"
     return {
@@ -116,10 +151,11 @@ def check_gather(w, grp, gpu, layers=None):
                 raise AssertionError(f"layer {layer} {name}: first mismatch at {tuple(bad)}")
 
 
-def full_check(w, group=0, score_impl=binding.WKV_SCORE_AUTO, staged=False):
+def full_check(w, group=0, score_impl=binding.WKV_SCORE_AUTO, staged=False, given_lse=False):
     grp = wl.make_group(w, group)
     ref = oracle.select_leader(grp["q_obs"], grp["k_layers"][0], **oracle_kwargs(w, grp))
-    gpu = run_gpu_group(w, grp, score_impl=score_impl, staged=staged)
+    gpu = run_gpu_group(w, grp, score_impl=score_impl, staged=staged,
+                        lse_obs=lse_obs_reference(w, grp) if given_lse else None)
     stats = check_selection(w, grp, gpu, ref)
     check_gather(w, grp, gpu)
     return grp, ref, gpu, stats

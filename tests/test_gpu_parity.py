@@ -67,6 +67,36 @@ def test_group_small(case, impl):
                 assert set(planted) <= set(gpu["window_idx"][b, h, :k].tolist())
 
 
+# ------------------------------------------------------------------ normalisers supplied by the caller
+@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("case", [
+    dict(),
+    dict(task=wl.TASK_AGGREGATION, top_p=31, window=32, l_obs=32),   # R = 128
+    dict(n_q_heads=8, n_kv_heads=1, l_obs=32, max_seqlen=2100),       # R = 256
+    dict(head_dim=64, window=4, l_obs=8),
+    dict(n_q_heads=6, n_kv_heads=2, l_obs=5, window=7, max_seqlen=999),
+    dict(dtype="f32", head_dim=64, n_q_heads=4, l_obs=8),
+    dict(ragged=True, batch=4, max_seqlen=1500),
+], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()) or "base")
+def test_group_with_given_normalisers(case, staged, impl):
+    """wkv_compress_group_lse / wkv_score_windows_lse: the log-sum-exp of every observation row comes
+    from the caller (computed here in float64 numpy from Eq. 1's definition); the result must meet
+    the same bars against the oracle as the self-contained path."""
+    w = small(**case)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=impl_for(w, impl), staged=staged, given_lse=True)
+    assert max_rel < 1e-4
+
+
+def test_given_normalisers_need_a_pointer():
+    w = small()
+    prob = binding.Problem.from_workload(w)
+    z = torch.zeros(16, device="cuda")
+    with pytest.raises(binding.WkvError) as e:
+        binding.wkv_score_windows_lse(prob, z, z, None, z, None, prob.alloc_workspace())
+    assert e.value.status == 1
+
+
 @pytest.mark.parametrize("impl", ["simt", "tc"])
 def test_stage_entry_points_and_token_scores(impl):
     w = small(max_seqlen=1100)
@@ -324,6 +354,10 @@ def test_config3_llama8b_32k(group):
     w = wl.llama8b_full()
     grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=group)
     assert gpu["prob"].k_max == 243 and gpu["prob"].keep_max == 3920
+
+
+def test_config3_with_given_normalisers():
+    pu.full_check(wl.llama8b_full(), group=2, given_lse=True)
 
 
 @pytest.mark.parametrize("n,depth", [(4096, 0.1), (16384, 0.5), (32768, 0.9)])
