@@ -598,10 +598,12 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             im.reuse = im.unit == s1_unit && im.chunk == s1_chunk && it == s1_it && im.n_tiles == s1_tiles &&
                        im.n_tiles >= kStages && im.chunk * len1 == im.j_begin;
             if (warp == 0) {
-                const int held = im.reuse ? kStages : 0;
-                if (lane == 0) produce(im, 0, held);
+                // ahead of the small loads of this item: the tiles the ring still holds (no traffic), or,
+                // when this is the only sweep, the first tiles from HBM as in sweep 1
+                const int ahead = im.reuse ? kStages : (a.lse_obs ? min(kEarlyTiles, im.n_tiles) : 0);
+                if (lane == 0) produce(im, 0, ahead);
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
-                if (lane == 0) produce(im, held, im.n_tiles);
+                if (lane == 0) produce(im, ahead, im.n_tiles);
             } else {
                 load_q_image(im, false);
                 if (warp == 1) {
