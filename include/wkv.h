@@ -229,6 +229,23 @@ int wkv_compress_group_lse(const wkv_shape *s, int32_t n_layers, const void *q_o
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Layer-by-layer use (section 2.2.2: the leader's indices serve the whole group).  During prefill
+ * the layers of a group appear one after the other: call this on the leader layer as soon as its
+ * keys exist (scores, pooling and selection in one launch on the tensor-core path, nothing
+ * gathered), keep window_idx, and call wkv_gather_kv with n_layers = 1 on the leader and on every
+ * follower layer when its K/V have been written.  The result equals wkv_compress_group on the
+ * same tensors.
+ *   lse_obs        DEVICE float [B, H_q, alpha] as in wkv_score_windows_lse, or NULL (then the
+ *                  normalisers are computed here)
+ *   window_scores  DEVICE out or NULL (then the scores live in the workspace only)
+ *   window_idx, kept_len, workspace   as in wkv_compress_group
+ */
+int wkv_select_leader_windows(const wkv_shape *s, const void *q_obs_leader, const void *k_leader,
+                              const float *lse_obs, float *window_scores,
+                              int32_t *window_idx, int32_t *kept_len,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The same group with every tensor in HOST memory (pinned memory recommended): the
  * inputs are copied to caller-provided DEVICE staging buffers, the group is
  * compressed there, and indices, kept lengths and the compact caches are copied

@@ -24,7 +24,8 @@ WKV_MAX_GROUP_LAYERS = 32
 EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
-    "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
+    "wkv_select_leader_windows", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
 
@@ -104,6 +105,8 @@ def lib() -> ctypes.CDLL:
     L.wkv_score_windows_lse.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.wkv_compress_group_lse.restype = ctypes.c_int
     L.wkv_compress_group_lse.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.wkv_select_leader_windows.restype = ctypes.c_int
+    L.wkv_select_leader_windows.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.wkv_compress_group_host.restype = ctypes.c_int
     L.wkv_compress_group_host.argtypes = [sp, i32, vp, sz, vp, vp, sz, vp, vp, sz, vp, vp,
                                           vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
@@ -288,6 +291,16 @@ def wkv_score_windows_lse(prob: Problem, q_obs, k_leader, lse_obs, window_scores
     _check(lib().wkv_score_windows_lse(ctypes.byref(prob.shape), _ptr(q_obs), _ptr(k_leader), _ptr(lse_obs),
                                        _ptr(window_scores), _ptr(token_scores), _ptr(workspace), workspace.numel(),
                                        _stream(stream)), "wkv_score_windows_lse")
+
+
+def wkv_select_leader_windows(prob: Problem, q_obs_leader, k_leader, window_scores, window_idx, kept_len, workspace,
+                              lse_obs=None, stream=None) -> None:
+    """Layer-by-layer use: score + pool + select on the leader layer only; the layers of the group are
+    then gathered one by one with wkv_gather_kv as their K/V appear."""
+    _check(lib().wkv_select_leader_windows(ctypes.byref(prob.shape), _ptr(q_obs_leader), _ptr(k_leader),
+                                           _ptr(lse_obs), _ptr(window_scores), _ptr(window_idx), _ptr(kept_len),
+                                           _ptr(workspace), workspace.numel(), _stream(stream)),
+           "wkv_select_leader_windows")
 
 
 def _group_lse_args(prob, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers, window_scores,

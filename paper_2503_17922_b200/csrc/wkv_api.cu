@@ -387,6 +387,26 @@ int wkv_score_windows_lse(const wkv_shape *s, const void *q_obs, const void *k_l
                                cuda_stream);
 }
 
+int wkv_select_leader_windows(const wkv_shape *s, const void *q_obs_leader, const void *k_leader,
+                              const float *lse_obs, float *window_scores, int32_t *window_idx, int32_t *kept_len,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!q_obs_leader || !k_leader || !window_idx || !kept_len) {
+        set_error_detail("q_obs_leader / k_leader / window_idx / kept_len is NULL");
+        return WKV_ERR_NULL;
+    }
+    const Workspace ws = plan_workspace(ks);
+    st = check_workspace(ws, workspace, workspace_bytes);
+    if (st != WKV_OK) return st;
+    float *scores = window_scores ? window_scores
+                                  : reinterpret_cast<float *>(static_cast<char *>(workspace) + ws.scores_off);
+    return do_score(s, ks, ws, q_obs_leader, k_leader, scores, nullptr, window_idx, kept_len, workspace,
+                    static_cast<cudaStream_t>(cuda_stream), lse_obs);
+}
+
 int wkv_select_topk_windows(const wkv_shape *s, const float *window_scores, int32_t *window_idx,
                             int32_t *kept_len, void *cuda_stream)
 {

@@ -88,6 +88,35 @@ def test_group_with_given_normalisers(case, staged, impl):
     assert max_rel < 1e-4
 
 
+@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("given_lse", [False, True])
+def test_layer_by_layer_use_equals_the_group_call(given_lse, impl):
+    """The leader is scored and selected alone, then every layer of the group is gathered by its own
+    call, as a prefill that produces the layers one after the other would do it."""
+    w = small(n_layers=3, gamma=3, task=wl.TASK_AGGREGATION, top_p=3)
+    grp = wl.make_group(w, 0)
+    lse_host = pu.lse_obs_reference(w, grp) if given_lse else None
+    ref = pu.run_gpu_group(w, grp, score_impl=IMPLS[impl], lse_obs=lse_host)
+    prob = binding.Problem.from_workload(w, score_impl=IMPLS[impl])
+    q = binding.to_device(grp["q_obs"])
+    out = prob.alloc_outputs(w.gamma, fill_byte=pu.FILL_BYTE)
+    work = prob.alloc_workspace()
+    lse = torch.from_numpy(lse_host).cuda() if given_lse else None
+    k0 = binding.to_device(grp["k_layers"][0])
+    binding.wkv_select_leader_windows(prob, q, k0, None, out["window_idx"], out["kept_len"], work, lse_obs=lse)
+    for l in range(w.gamma):                                   # the layers arrive one at a time
+        k, v = binding.to_device(grp["k_layers"][l]), binding.to_device(grp["v_layers"][l])
+        binding.wkv_gather_kv(prob, [k], [v], out["window_idx"], [out["k_out"][l]], [out["v_out"][l]],
+                              keep_capacity=out["keep_capacity"])
+    torch.cuda.synchronize()
+    assert binding.device_status(work) == 0
+    np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), ref["window_idx"])
+    np.testing.assert_array_equal(out["kept_len"].cpu().numpy(), ref["kept_len"])
+    for l in range(w.gamma):
+        np.testing.assert_array_equal(binding.to_host_bits(out["k_out"][l]), ref["k_out"][l])
+        np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][l]), ref["v_out"][l])
+
+
 def test_given_normalisers_need_a_pointer():
     w = small()
     prob = binding.Problem.from_workload(w)
