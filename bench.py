@@ -244,13 +244,18 @@ def main() -> None:
     gather_calls = [binding.prepare_gather_kv(prob, d["k"], d["v"], out["window_idx"], out["k_out"], out["v_out"],
                                               keep_capacity=cap, stream=stream) for d in dev_groups]
 
+    # the call of the timed loop: the group recorded once per resident group (wkv_group_plan_create),
+    # replayed with wkv_group_plan_launch, as an engine with static buffers would issue it
+    plans = [binding.GroupPlan(prob, d["q"], d["k"], d["v"], out["k_out"], out["v_out"], out["window_scores"],
+                               out["window_idx"], out["kept_len"], work, keep_capacity=cap) for d in dev_groups]
+
     barrier = replicas.barrier
 
     with torch.cuda.stream(stream):
         for i in range(warmup):
             if flush is not None:
                 flush.fill_(i & 0xFF)
-            group_calls[i % n_groups].run()
+            plans[i % n_groups].launch(stream)
         barrier()
         sampler = ClockSampler(local)
         if rank == 0:
@@ -260,7 +265,7 @@ def main() -> None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             for i in range(args.steps):
-                group_calls[i % n_groups].run()
+                plans[i % n_groups].launch(stream)
             e1.record(stream)
             barrier()
             ms_total = e0.elapsed_time(e1)
@@ -270,7 +275,7 @@ def main() -> None:
             for i in range(args.steps):
                 flush.fill_(i & 0xFF)
                 evs[i][0].record(stream)
-                group_calls[i % n_groups].run()
+                plans[i % n_groups].launch(stream)
                 evs[i][1].record(stream)
             barrier()
             ms_total = sum(a.elapsed_time(b) for a, b in evs)
@@ -319,6 +324,17 @@ def main() -> None:
             stream.synchronize()
             return a.elapsed_time(b) / (reps * n)
 
+        # the same group through the direct entry point, call by call (two launches on the stream per step)
+        ms_direct = None
+        if flush is None:
+            n_direct = min(args.steps, 1000)
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            d0.record(stream)
+            for i in range(n_direct):
+                group_calls[i % n_groups].run()
+            d1.record(stream)
+            stream.synchronize()
+            ms_direct = d0.elapsed_time(d1) / n_direct
         ms_fused = time_stage(group_calls)                 # score+select kernel followed by the gather kernel
         ms_score = time_stage(score_calls)                 # the same kernel without the selection
         ms_select = time_stage([select_call])              # stand-alone selection kernel (not on the fused path)
@@ -403,6 +419,7 @@ def main() -> None:
             "config": {"workload": w.name, "batch": w.batch, "seq_len": w.max_seqlen, "layers_per_group": w.gamma,
                        "groups_rotated": n_groups, "l_obs": w.l_obs, "window": w.window,
                        "budget_tokens": int(w.budgets()[0]), "score_impl": args.score_impl,
+                       "call": "wkv_group_plan_launch (one recorded group per step)",
                        "cold_cache": "flush of 256 MB between steps" if flush is not None
                        else f"{n_groups} groups rotated ({resident / 1e9:.2f} GB resident, larger than L2)"},
             "gpu_launches": int(launches),
@@ -410,7 +427,8 @@ def main() -> None:
             "path_algorithmic_bytes": alg["total"],
             "stages_ms": {"group_graph_replay": ms_fused, "score_select_fused": ms_score_select,
                           "score_only": ms_score, "select_standalone": ms_select, "gather": ms_gather,
-                          "group_given_lse_graph_replay": ms_given_lse},
+                          "group_given_lse_graph_replay": ms_given_lse,
+                          "group_direct_call": ms_direct},
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "clocks": clocks,
         }))
     replicas.shutdown()

@@ -246,6 +246,33 @@ int wkv_select_leader_windows(const wkv_shape *s, const void *q_obs_leader, cons
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * A layer group as a replayable object (sections 2.2.1-2.2.2, the same computation as
+ * wkv_compress_group / wkv_compress_group_lse).  For engines that call the group with the same
+ * buffers again and again (static K/V pools and compact caches): create records the launches of
+ * the call in a CUDA graph once, launch replays it on a stream, which leaves a smaller gap at the
+ * kernel boundary than separate launches do.  The plan owns only the graph; every buffer stays
+ * the caller's and must stay valid and at its address for as long as the plan is launched.  What a
+ * launch computes depends on the buffers' contents at that moment only.
+ *   create   arguments as wkv_compress_group_lse (lse_obs may be NULL: then the normalisers are
+ *            computed); validates as the direct call does and launches nothing.  Host-side
+ *            resources (a graph) are allocated; no device buffer of the caller's is touched.
+ *            `budgets` and the strides of `s` are read now, not at launch.
+ *   launch   enqueues the group on cuda_stream; one plan is in flight once at a time (it uses
+ *            the one workspace it was created with).
+ *   destroy  after the last launch has completed.  NULL is ignored.
+ */
+typedef struct wkv_group_plan wkv_group_plan;
+int wkv_group_plan_create(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
+                          const float *lse_obs,
+                          const void *const *k_layers, const void *const *v_layers,
+                          void *const *k_out_layers, void *const *v_out_layers,
+                          float *window_scores, int32_t *window_idx, int32_t *kept_len,
+                          const int32_t *cu_seqlens_out, int32_t keep_capacity,
+                          void *workspace, size_t workspace_bytes, wkv_group_plan **plan_out);
+int wkv_group_plan_launch(wkv_group_plan *plan, void *cuda_stream);
+void wkv_group_plan_destroy(wkv_group_plan *plan);
+
+/*
  * The same group with every tensor in HOST memory (pinned memory recommended): the
  * inputs are copied to caller-provided DEVICE staging buffers, the group is
  * compressed there, and indices, kept lengths and the compact caches are copied

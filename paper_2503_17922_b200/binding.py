@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
-    "wkv_select_leader_windows", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_select_leader_windows", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
 
@@ -107,6 +107,13 @@ def lib() -> ctypes.CDLL:
     L.wkv_compress_group_lse.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     L.wkv_select_leader_windows.restype = ctypes.c_int
     L.wkv_select_leader_windows.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.wkv_group_plan_create.restype = ctypes.c_int
+    L.wkv_group_plan_create.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz,
+                                        ctypes.POINTER(vp)]
+    L.wkv_group_plan_launch.restype = ctypes.c_int
+    L.wkv_group_plan_launch.argtypes = [vp, vp]
+    L.wkv_group_plan_destroy.restype = None
+    L.wkv_group_plan_destroy.argtypes = [vp]
     L.wkv_compress_group_host.restype = ctypes.c_int
     L.wkv_compress_group_host.argtypes = [sp, i32, vp, sz, vp, vp, sz, vp, vp, sz, vp, vp,
                                           vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
@@ -319,6 +326,39 @@ def wkv_compress_group_lse(prob: Problem, q_obs_leader, lse_obs, k_layers, v_lay
                                   window_scores, window_idx, kept_len, workspace, cu_seqlens_out, keep_capacity,
                                   stream)
     _check(lib().wkv_compress_group_lse(*args), "wkv_compress_group_lse")
+
+
+class GroupPlan:
+    """wkv_group_plan: the group call recorded once, replayed by `launch(stream)`.  Keeps the tensors
+    it was created with alive."""
+
+    def __init__(self, prob: Problem, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers, window_scores,
+                 window_idx, kept_len, workspace, lse_obs=None, cu_seqlens_out=None, keep_capacity: int = 0):
+        args, arrs = _group_lse_args(prob, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                                     window_scores, window_idx, kept_len, workspace, cu_seqlens_out, keep_capacity,
+                                     None)
+        self._keep = (prob, arrs, q_obs_leader, lse_obs, k_layers, v_layers, k_out_layers, v_out_layers,
+                      window_scores, window_idx, kept_len, workspace, cu_seqlens_out)
+        handle = ctypes.c_void_p()
+        _check(lib().wkv_group_plan_create(*args[:-1], ctypes.byref(handle)), "wkv_group_plan_create")
+        self._handle = handle
+        self._launch = lib().wkv_group_plan_launch
+
+    def launch(self, stream=None) -> None:
+        st = self._launch(self._handle, _stream(stream))
+        if st != 0:
+            _check(st, "wkv_group_plan_launch")
+
+    def close(self) -> None:
+        if self._handle:
+            lib().wkv_group_plan_destroy(self._handle)
+            self._handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class PreparedCall:

@@ -446,7 +446,13 @@ int wkv_gather_kv(const wkv_shape *s, int32_t n_layers, const void *const *k_lay
                       "gather kernel");
 }
 
-static int compress_group_entry(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader, const float *lse_obs,
+}  // extern "C"
+
+namespace wkv {
+uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+}  // namespace wkv
+
+int wkv::compress_group_entry(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader, const float *lse_obs,
                                 const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
                                 void *const *v_out_layers, float *window_scores, int32_t *window_idx,
                                 int32_t *kept_len, const int32_t *cu_seqlens_out, int32_t keep_capacity,
@@ -480,6 +486,8 @@ static int compress_group_entry(const wkv_shape *s, int32_t n_layers, const void
                                     keep_capacity, stream),
                       "gather kernel");
 }
+
+extern "C" {
 
 int wkv_compress_group(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader,
                        const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,

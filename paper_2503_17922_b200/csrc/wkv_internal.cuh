@@ -182,6 +182,13 @@ int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const vo
              cudaStream_t stream, const float *lse_obs = nullptr);
 
 void count_launches(int n);
+uint64_t launches_so_far();
+// the group call behind wkv_compress_group / wkv_compress_group_lse (lse_obs may be null)
+int compress_group_entry(const wkv_shape *s, int32_t n_layers, const void *q_obs_leader, const float *lse_obs,
+                         const void *const *k_layers, const void *const *v_layers, void *const *k_out_layers,
+                         void *const *v_out_layers, float *window_scores, int32_t *window_idx, int32_t *kept_len,
+                         const int32_t *cu_seqlens_out, int32_t keep_capacity, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream);
 void set_error_detail(const char *fmt, ...);
 
 }  // namespace wkv

@@ -117,6 +117,47 @@ def test_layer_by_layer_use_equals_the_group_call(given_lse, impl):
         np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][l]), ref["v_out"][l])
 
 
+def test_group_plan_replays_the_group_call():
+    """A recorded group must give what the direct call gives, on whatever the buffers hold at launch."""
+    w = small(task=wl.TASK_AGGREGATION, top_p=31, window=32, l_obs=32)
+    prob = binding.Problem.from_workload(w)
+    grps = [wl.make_group(w, 0), wl.make_group(wl.scaled(w, config_id=10), 0)]
+    q = binding.to_device(grps[0]["q_obs"])
+    ks = [binding.to_device(x) for x in grps[0]["k_layers"]]
+    vs = [binding.to_device(x) for x in grps[0]["v_layers"]]
+    out = prob.alloc_outputs(w.gamma, fill_byte=pu.FILL_BYTE)
+    work = prob.alloc_workspace()
+    n0 = binding.wkv_launch_count()
+    plan = binding.GroupPlan(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
+                             out["kept_len"], work, keep_capacity=out["keep_capacity"])
+    assert binding.wkv_launch_count() == n0          # recording launches nothing
+    for grp in grps + grps[:1]:                       # new contents in the same buffers, then the first again
+        q.copy_(binding.to_device(grp["q_obs"]))
+        for dst, src in zip(ks + vs, grp["k_layers"] + grp["v_layers"]):
+            dst.copy_(binding.to_device(src))
+        before = binding.wkv_launch_count()
+        plan.launch()
+        torch.cuda.synchronize()
+        assert binding.wkv_launch_count() - before >= 2
+        assert binding.device_status(work) == 0
+        ref = pu.run_gpu_group(w, grp)
+        np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), ref["window_idx"])
+        np.testing.assert_array_equal(out["kept_len"].cpu().numpy(), ref["kept_len"])
+        for l in range(w.gamma):
+            kept = ref["kept_len"]
+            for b in range(w.batch):
+                for h in range(w.n_kv_heads):
+                    n_keep = int(kept[b, h])
+                    np.testing.assert_array_equal(binding.to_host_bits(out["k_out"][l])[b, h, :n_keep],
+                                                  ref["k_out"][l][b, h, :n_keep])
+                    np.testing.assert_array_equal(binding.to_host_bits(out["v_out"][l])[b, h, :n_keep],
+                                                  ref["v_out"][l][b, h, :n_keep])
+    plan.close()
+    with pytest.raises(binding.WkvError):
+        binding.GroupPlan(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
+                          out["kept_len"], work, keep_capacity=1)          # refused at creation, as by the direct call
+
+
 def test_given_normalisers_need_a_pointer():
     w = small()
     prob = binding.Problem.from_workload(w)
