@@ -179,7 +179,9 @@ int wkv_select_topk_windows(const wkv_shape *s, const float *window_scores,
  * followed by the observation rows n-alpha .. n-1.  Bit copies.
  *   k_layers, v_layers          HOST arrays [n_layers] of DEVICE pointers (inputs, layout of `s`)
  *   k_out_layers, v_out_layers  HOST arrays [n_layers] of DEVICE pointers (outputs)
- *   window_idx                  DEVICE int32 [B, H_kv, wkv_k_max()] as written by the selection
+ *   window_idx                  DEVICE int32 [B, H_kv, wkv_k_max()] as written by the selection; an entry
+ *                               outside [0, K_w) among a unit's first k is skipped (its rows of the
+ *                               output are left as they are), never followed
  *   cu_seqlens_out              DEVICE int32 [B+1] or NULL.
  *       NULL  => dense output [B, H_kv, keep_capacity, d]; rows >= kept_len are not written.
  *       else  => packed output [T_out, H_kv, d], sequence b starting at row cu_seqlens_out[b].

@@ -85,7 +85,11 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
     for (int slot = blockIdx.x * prm.slots_per_block + warp; slot < slot_end; slot += kWarps) {
         int src_row0, dst_row0, n_rows;
         if (slot < k) {
-            src_row0 = idx[slot] * s.omega;
+            // an entry that is no window of this sequence (a list that no selection has written, or
+            // that the caller filled wrongly) is skipped: the kernel never leaves the tensors
+            const int wi = idx[slot];
+            if (wi < 0 || wi >= kw) continue;
+            src_row0 = wi * s.omega;
             n_rows = min(s.omega, n_r - src_row0);
             dst_row0 = slot * s.omega;
         } else {

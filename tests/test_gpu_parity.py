@@ -158,6 +158,35 @@ def test_group_plan_replays_the_group_call():
                           out["kept_len"], work, keep_capacity=1)          # refused at creation, as by the direct call
 
 
+def test_expired_wait_sets_the_status_word_and_the_context_survives():
+    """Every wait inside the fused kernel is bounded.  Here the arrival count of unit 0 is set so far
+    below zero that it can never reach its target: the blocks of that unit give up after about a
+    second, the kernel ends, bit 0 of the status word is set, and after zeroing the workspace the
+    same call works again.  (Workspace layout: status word at byte 0, per unit u a ticket and an
+    arrival word at int32 index 16 + 16 + 2u and the one after it.)"""
+    w = small()
+    prob = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05)
+    grp = wl.make_group(w, 0)
+    q = binding.to_device(grp["q_obs"])
+    ks = [binding.to_device(x) for x in grp["k_layers"]]
+    vs = [binding.to_device(x) for x in grp["v_layers"]]
+    out = prob.alloc_outputs(len(ks), fill_byte=pu.FILL_BYTE)
+    work = prob.alloc_workspace()
+    words = work[:4096].view(torch.int32)
+    words[16 + 16 + 1] = -1000000
+    binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
+                               out["kept_len"], work, keep_capacity=out["keep_capacity"])
+    torch.cuda.synchronize()                      # returns: nothing hangs
+    assert binding.device_status(work) & 1
+    work.zero_()
+    gpu = pu.run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_TCGEN05)
+    binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
+                               out["kept_len"], work, keep_capacity=out["keep_capacity"])
+    torch.cuda.synchronize()
+    assert binding.device_status(work) == 0
+    np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), gpu["window_idx"])
+
+
 def test_given_normalisers_need_a_pointer():
     w = small()
     prob = binding.Problem.from_workload(w)
@@ -337,6 +366,40 @@ def test_gather_with_given_indices(dtype, d, packed_out):
     for layer in range(w.gamma):
         np.testing.assert_array_equal(binding.to_host_bits(outs[0][layer]), oracle.gather_layer(grp["k_layers"][layer], idx, **kw_))
         np.testing.assert_array_equal(binding.to_host_bits(outs[1][layer]), oracle.gather_layer(grp["v_layers"][layer], idx, **kw_))
+
+
+def test_gather_skips_entries_that_are_no_window():
+    """A list that no selection has written (here: garbage in one unit) must not take the gather out of
+    the tensors: such entries are skipped, their output rows keep the fill, every other unit and the
+    observation rows are copied as usual."""
+    w = small(n_layers=1, gamma=1)
+    grp = wl.make_group(w, 0)
+    prob = binding.Problem.from_workload(w)
+    ref = oracle.select_leader(grp["q_obs"], grp["k_layers"][0], **pu.oracle_kwargs(w, grp))
+    idx = np.array(ref["window_idx"], dtype=np.int32).reshape(w.batch, w.n_kv_heads, prob.k_max).copy()
+    good = idx.copy()
+    idx[0, 1, :] = np.int32(-1515870811)              # 0xA5A5A5A5: an output buffer nobody wrote
+    idx[1, 0, 0] = 2 ** 30                             # far beyond the last window
+    k_dev = binding.to_device(grp["k_layers"][0])
+    cap = prob.keep_max
+    tdt = torch.bfloat16
+    outs = []
+    for table in (idx, good):
+        o = torch.empty((w.batch, w.n_kv_heads, cap, w.head_dim), dtype=tdt, device="cuda")
+        o.view(torch.uint8).fill_(pu.FILL_BYTE)
+        binding.wkv_gather_kv(prob, [k_dev], None, torch.from_numpy(table).cuda(), [o], None, keep_capacity=cap)
+        outs.append(binding.to_host_bits(o))
+    torch.cuda.synchronize()
+    bad, ok = outs
+    fill = pu.fill_pattern(w.dtype)
+    np.testing.assert_array_equal(bad[0, 0], ok[0, 0])                       # untouched units
+    np.testing.assert_array_equal(bad[1, 1], ok[1, 1])
+    k = oracle.num_selected(int(grp["seqlens"][0]), w.l_obs, w.window, int(grp["budgets"][0]))
+    assert (bad[0, 1, : k * w.window] == fill).all()                         # every slot of the garbage unit skipped
+    np.testing.assert_array_equal(bad[0, 1, k * w.window: k * w.window + w.l_obs],
+                                  ok[0, 1, k * w.window: k * w.window + w.l_obs])   # observation rows still copied
+    assert (bad[1, 0, : w.window] == fill).all()                             # the one bad slot skipped ...
+    np.testing.assert_array_equal(bad[1, 0, w.window:], ok[1, 0, w.window:])  # ... the rest as usual
 
 
 # ------------------------------------------------------------------ degenerate cases
