@@ -16,10 +16,11 @@
 // Units are taken in waves whose keys fit L2 together.  A work item is (unit, chunk of <= 17 key
 // tiles); the persistent blocks (at most one per SM) take the items of a wave round-robin.
 //
-// Warp roles: warp 0 issues the TMA tile loads (4-stage ring), warp 1 issues the MMAs into NG
-// accumulator buffers in tensor memory, and NG compute groups of four warps (one warp per 32-lane
-// quarter of tensor memory) take the tiles round-robin, each with its own buffer, 32 columns at a
-// time; the four warps that share an SM sub-partition cover each other's load latency.  The
+// Warp roles: warp 0 issues the TMA tile loads (4-stage ring), warp 1 issues the MMAs into four
+// accumulator buffers of 128 columns in tensor memory, and four compute groups of four warps (one
+// warp per 32-lane quarter of tensor memory) take the accumulators round-robin, each with its own
+// buffer, 32 columns at a time.  With more than 128 observation rows (up to 256) every key tile
+// gives two accumulators, one per 128-row block of Q, which go through the same buffers and groups; the four warps that share an SM sub-partition cover each other's load latency.  The
 // contraction is the only tensor-core work; exponentials, sums and pooling are fp32 on the CUDA
 // cores in a fixed order, so results are bit-identical from run to run.
 //
@@ -43,7 +44,7 @@ using namespace tc;
 constexpr int kStages = 4;
 constexpr int kEarlyTiles = 2;                           // key tiles requested ahead of the Q image at the start of an item
 constexpr int kMaxGroups = 4;
-__host__ __device__ constexpr int groups_for(int mb) { return mb == 1 ? 4 : 2; }
+__host__ __device__ constexpr int groups_for(int) { return 4; }
 __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for(mb) * 128; }
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
@@ -260,7 +261,11 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     constexpr int kThreads = block_threads(MB);
     constexpr int q_rows = MB * 128;
     constexpr int q_region = q_rows * 128;                // bytes of one 64-column block of the Q image
-    constexpr uint32_t buf_cols = MB * 128;               // accumulator buffer stride in tensor memory
+    // A key tile gives one accumulator of 128 columns per 128-row block of Q ("half" rh = 0, 1 with
+    // two row blocks); accumulators are numbered v = tile * MB + rh across the block's whole tile
+    // stream, and buffers and compute groups take them round-robin (v mod NG).  With two row blocks a
+    // group therefore always works on the same half (NG is even).
+    constexpr uint32_t buf_cols = 128;                    // accumulator buffer stride in tensor memory
     constexpr uint32_t tmem_cols = 512;
     static_assert(NG * buf_cols <= tmem_cols, "accumulator buffers exceed tensor memory");
 
@@ -269,9 +274,9 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ int flag_s;
-    __shared__ float2 part[NG][MB][128];
-    __shared__ __align__(16) float neg_lse2[256];        // -log2 of the row normaliser; -inf for padding rows
-    __shared__ float t_chunk[kChunkCap];
+    __shared__ float2 part[NG][1][128];                    // sweep 1: a group's (max, sum) of the rows on its lanes
+    __shared__ __align__(16) float neg_lse2_all[256];    // -log2 of the row normaliser; -inf for padding rows
+    __shared__ float t_chunk[MB][kChunkCap];              // sweep 2: per half, the key's sum over that half's rows
     __shared__ TopkSmem topk_sm;
 
     const KShape &s = a.s;
@@ -396,47 +401,47 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         }
     };
 
-    // MMA issue for one item.  sweep 1: D[rows, keys] = Q K^T (MB row blocks); sweep 2: D[keys, rows] = K Q^T.
+    // MMA issue for one item.  sweep 1: D[rows, keys] = Q K^T; sweep 2: D[keys, rows] = K Q^T; per key
+    // tile one accumulator per 128-row block of Q.
     // One thread issues everything, so its instruction count per tile is on the critical path: the
     // matrix descriptors of Q and of stage 0 are built once, and every k-step only adds a
     // compile-time constant to the address field (the fields above it never change).
     const uint64_t q_desc0 = umma_desc_sw128(smem_u32(q_img));
     const uint64_t k_desc0 = umma_desc_sw128(smem_u32(k_stage0));
-    auto issue_tile = [&](auto ksteps_tag, uint32_t d_tmem, uint64_t k_desc, uint32_t idesc, bool sweep2) {
+    auto issue_tile = [&](auto ksteps_tag, uint32_t d_tmem, uint64_t k_desc, uint64_t q_desc, uint32_t idesc,
+                          bool sweep2) {
         constexpr int KSTEPS = decltype(ksteps_tag)::value;
-        if (sweep2) {
 #pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                const uint32_t qo = (uint32_t)((ks >> 2) * q_region + (ks & 3) * 32) >> 4;
-                const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
-                umma_bf16(d_tmem, k_desc + ko, q_desc0 + qo, idesc, ks > 0);
-            }
-        } else {
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                for (int ks = 0; ks < KSTEPS; ++ks) {
-                    const uint32_t qo = (uint32_t)((ks >> 2) * q_region + mb * kRegion + (ks & 3) * 32) >> 4;
-                    const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
-                    umma_bf16(d_tmem + mb * 128, q_desc0 + qo, k_desc + ko, idesc, ks > 0);
-                }
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            const uint32_t qo = (uint32_t)((ks >> 2) * q_region + (ks & 3) * 32) >> 4;
+            const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
+            if (sweep2) umma_bf16(d_tmem, k_desc + ko, q_desc + qo, idesc, ks > 0);
+            else umma_bf16(d_tmem, q_desc + qo, k_desc + ko, idesc, ks > 0);
         }
     };
     auto issue_mma = [&](const Item &im, bool sweep2) {
-        const uint32_t idesc = sweep2 ? umma_idesc_bf16(128, a.r16) : umma_idesc_bf16(128, kTile);
         const uint32_t stage_step = (uint32_t)stage_bytes >> 4;
         for (int t = 0; t < im.n_tiles; ++t) {
             const uint32_t g = it + t;
-            const int st = g % kStages, buf = g % NG;
+            const int st = g % kStages;
             if (!mbar_wait(&bar.full[st], (g / kStages) & 1, &abort_s)) return;
-            if (g >= NG && !mbar_wait(&bar.tempty[buf], ((g / NG) - 1) & 1, &abort_s)) return;
-            tc_fence_after_sync();
             const uint64_t k_desc = k_desc0 + (uint64_t)(st * stage_step);
-            const uint32_t d_tmem = tmem_base + buf * buf_cols;
-            if (ksteps == 8) issue_tile(std::integral_constant<int, 8>{}, d_tmem, k_desc, idesc, sweep2);
-            else issue_tile(std::integral_constant<int, 4>{}, d_tmem, k_desc, idesc, sweep2);
+#pragma unroll
+            for (int rh = 0; rh < MB; ++rh) {
+                const uint32_t v = g * MB + rh;
+                const int buf = v % NG;
+                if (v >= NG && !mbar_wait(&bar.tempty[buf], ((v / NG) - 1) & 1, &abort_s)) return;
+                tc_fence_after_sync();
+                // sweep 2: the rows of this half are the N dimension (a multiple of 16)
+                const int n_rows = rh == 0 ? min(a.r16, 128) : a.r16 - 128;
+                const uint32_t idesc = sweep2 ? umma_idesc_bf16(128, n_rows) : umma_idesc_bf16(128, kTile);
+                const uint64_t q_desc = q_desc0 + (uint64_t)((rh * kRegion) >> 4);
+                const uint32_t d_tmem = tmem_base + buf * buf_cols;
+                if (ksteps == 8) issue_tile(std::integral_constant<int, 8>{}, d_tmem, k_desc, q_desc, idesc, sweep2);
+                else issue_tile(std::integral_constant<int, 4>{}, d_tmem, k_desc, q_desc, idesc, sweep2);
+                umma_commit(&bar.tfull[buf]);
+            }
             umma_commit(&bar.empty[st]);
-            umma_commit(&bar.tfull[buf]);
         }
     };
 
@@ -450,44 +455,45 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         const int col0 = MB == 2 ? 0 : (L / Rp) * Rp;       // warp-uniform: Rp is a multiple of 32
         const int gshift = ncols == 128 ? 2 : (ncols == 64 ? 1 : 0);   // log2(32-column groups per row block)
         const int gmask = (1 << gshift) - 1;
-        const int nslot = MB << gshift;
-        float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
-        int limit0, limit1 = -1;                            // last key each row may attend to
+        const int nslot = 1 << gshift;                      // 32-column slots of an accumulator this thread reduces
+        float m0 = -INFINITY, l0 = 0.f;
+        int limit0;                                         // last key the thread's row may attend to
         {
-            const int row = MB == 2 ? L : L % Rp;
+            const int row = MB == 2 ? (grp & 1) * 128 + L : L % Rp;
             limit0 = row < s.R ? min(im.n_r + row % s.alpha, im.j_end - 1) : -1;
-            if (MB == 2) limit1 = 128 + L < s.R ? min(im.n_r + (128 + L) % s.alpha, im.j_end - 1) : -1;
         }
         const uint32_t taddr = taddr_grp + col0;
-        for (int t = 0; t < im.n_tiles; ++t) {
-            const uint32_t g = it + t;
-            if ((int)(g % NG) != grp) continue;
-            if (!warp_wait(&bar.tfull[grp], (g / NG) & 1, &abort_s, lane)) break;
+        (void)gmask;
+        for (uint32_t v = it * MB; v < (it + im.n_tiles) * MB; ++v) {
+            if ((int)(v % NG) != grp) continue;
+            const int t = (int)(v / MB - it);
+            if (!warp_wait(&bar.tfull[grp], (v / NG) & 1, &abort_s, lane)) break;
             tc_fence_after_sync();
             const int tile0 = im.j_begin + t * kTile;
             const int j0 = tile0 + col0;
             const bool fast = (tile0 + kTile - 1 <= im.n_r) && (tile0 + kTile - 1 < im.j_end);   // no masking
-            // slot sl = 32 columns: row block sl >> gshift, column group sl & gmask
             for (int sl = 0; sl < nslot; ++sl) {
-                float v[32];
-                tmem_ld32(taddr + (sl >> gshift) * 128 + (sl & gmask) * 32, v);
+                float x[32];
+                tmem_ld32(taddr + sl * 32, x);
                 if (sl + 1 == nslot) warp_release(&bar.tempty[grp], lane);   // the buffer may be overwritten now
-                if (MB == 2 && (sl >> gshift)) stats_update(v, fast, j0 + (sl & gmask) * 32, limit1, c, m1, l1);
-                else stats_update(v, fast, j0 + (sl & gmask) * 32, limit0, c, m0, l0);
+                stats_update(x, fast, j0 + sl * 32, limit0, c, m0, l0);
             }
         }
         part[grp][0][L] = make_float2(m0, l0);
-        if (MB == 2) part[grp][MB - 1][L] = make_float2(m1, l1);
     };
 
     // sweep-2 compute: token score of key L of every tile of the item -> t_chunk (and token_scores)
     auto compute_scores = [&](const Item &im) {
-        const int n32 = a.r16 >> 5;                  // 32-row groups; a 16-row tail follows if r16 & 16
-        const bool tail = (a.r16 & 16) != 0;
-        for (int t = 0; t < im.n_tiles; ++t) {
-            const uint32_t g = it + t;
-            if ((int)(g % NG) != grp) continue;
-            if (!warp_wait(&bar.tfull[grp], (g / NG) & 1, &abort_s, lane)) break;
+        // rows of the group's half: 32-row slices; a 16-row tail follows if their number has bit 4 set
+        const int rh = MB == 2 ? (grp & 1) : 0;
+        const int rows_h = rh == 0 ? min(a.r16, 128) : a.r16 - 128;
+        const int n32 = rows_h >> 5;
+        const bool tail = (rows_h & 16) != 0;
+        const float *neg_lse2 = neg_lse2_all + rh * 128;
+        for (uint32_t av = it * MB; av < (it + im.n_tiles) * MB; ++av) {
+            if ((int)(av % NG) != grp) continue;
+            const int t = (int)(av / MB - it);
+            if (!warp_wait(&bar.tfull[grp], (av / NG) & 1, &abort_s, lane)) break;
             tc_fence_after_sync();
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
             for (int sl = 0; sl < n32; ++sl) {
@@ -505,8 +511,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             const float tj = (a0 + a1) + (a2 + a3);
             const int j = im.j_begin + tile_at(im, t) * kTile + L;
             if (j < im.j_end) {
-                t_chunk[j - im.j_begin] = tj;
-                if (a.token_scores) a.token_scores[(size_t)im.unit * s.nr_max + j] = tj;
+                t_chunk[rh][j - im.j_begin] = tj;
+                if (MB == 1 && a.token_scores) a.token_scores[(size_t)im.unit * s.nr_max + j] = tj;
             }
         }
     };
@@ -558,14 +564,16 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 float2 res = make_float2(-INFINITY, 0.f);
                 if (r < s.R) {
                     const int mb = MB == 2 ? r >> 7 : 0, base = MB == 2 ? (r & 127) : r;
+                    // with two row blocks a row lives in the groups of its half (group index odd or even)
                     float M = -INFINITY;
                     for (int g = 0; g < NG; ++g)
-                        for (int cp = 0; cp < copies; ++cp) M = fmaxf(M, part[g][mb][base + cp * Rp].x);
+                        for (int cp = 0; cp < copies; ++cp)
+                            if (MB == 1 || (g & 1) == mb) M = fmaxf(M, part[g][0][base + cp * Rp].x);
                     float sum = 0.f;
                     for (int g = 0; g < NG; ++g)
                         for (int cp = 0; cp < copies; ++cp) {
-                            const float2 p = part[g][mb][base + cp * Rp];
-                            if (p.y > 0.f) sum += p.y * fast_exp2((p.x - M) * c);
+                            const float2 p = part[g][0][base + cp * Rp];
+                            if ((MB == 1 || (g & 1) == mb) && p.y > 0.f) sum += p.y * fast_exp2((p.x - M) * c);
                         }
                     res = make_float2(M * c, sum);
                 }
@@ -628,7 +636,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                             v = -1.4426950408889634f *
                                 __ldg(a.lse_obs + ((size_t)im.b * s.hq + (size_t)im.h * s.G + g) * s.alpha + i);
                         }
-                        neg_lse2[tl] = v;
+                        neg_lse2_all[tl] = v;
                     }
                     go_producer();
                     asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
@@ -681,7 +689,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                         }
                         if (sum > 0.f) v = -(M + log2f(sum));
                     }
-                    neg_lse2[tl] = v;
+                    neg_lse2_all[tl] = v;
                 }
                 asm volatile("bar.sync 3, %0;" ::"n"(kComputeThreads) : "memory");
                 compute_scores(im);
@@ -694,6 +702,16 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             __syncthreads();
             tc_fence_after_sync();
             if (abort_s) break;
+            float *t_item = &t_chunk[0][0];
+            if (MB == 2) {
+                // Eq. 2 sums over all rows: add the two halves' sums of every key
+                for (int x = threadIdx.x; x < im.j_end - im.j_begin; x += kThreads) {
+                    const float tj = t_chunk[0][x] + t_chunk[MB - 1][x];
+                    t_item[x] = tj;
+                    if (a.token_scores) a.token_scores[(size_t)im.unit * s.nr_max + im.j_begin + x] = tj;
+                }
+                __syncthreads();
+            }
             // Eq. 3-4: the item's windows (its first key is a multiple of omega)
             {
                 const int n_tok = im.j_end - im.j_begin;
@@ -705,17 +723,17 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                         const int lw = i;
                         const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
                         float r;
-                        if (s.omega == 16) r = pool_window_sorted<16>(t_chunk + lo, size, s.p);
-                        else if (s.omega == 8) r = pool_window_sorted<8>(t_chunk + lo, size, s.p);
-                        else if (s.omega == 32) r = pool_window_sorted<32>(t_chunk + lo, size, s.p);
-                        else r = pool_window_sorted<4>(t_chunk + lo, size, s.p);
+                        if (s.omega == 16) r = pool_window_sorted<16>(t_item + lo, size, s.p);
+                        else if (s.omega == 8) r = pool_window_sorted<8>(t_item + lo, size, s.p);
+                        else if (s.omega == 32) r = pool_window_sorted<32>(t_item + lo, size, s.p);
+                        else r = pool_window_sorted<4>(t_item + lo, size, s.p);
                         ws_out[lw] = r;
                     }
                 }
                 else {
                     for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
                         const int lo = lw * s.omega;
-                        ws_out[lw] = pool_top_p(t_chunk + lo, min(s.omega, n_tok - lo), s.p);
+                        ws_out[lw] = pool_top_p(t_item + lo, min(s.omega, n_tok - lo), s.p);
                     }
                 }
             }
