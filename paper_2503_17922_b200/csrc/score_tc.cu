@@ -126,27 +126,27 @@ __device__ __forceinline__ void red_release_gpu_add(int *p, int v)
 {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ bool warp_wait_arrivals(const int *word, int target, volatile int *abort_flag, int lane)
+// one thread: polls until the word has reached `target`; false once the block has given up
+__device__ __forceinline__ bool poll_until_at_least(const int *word, int target, volatile int *abort_flag)
 {
-    int ok = 1;
-    if (lane == 0) {
-        unsigned long long t0 = 0;
-        for (uint32_t spin = 1; ld_acquire_gpu(word) < target; ++spin) {
-            if (*abort_flag) {
-                ok = 0;
-                break;
-            }
-            if ((spin & 255u) == 0u) {
-                const unsigned long long now = global_timer_ns();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > 2 * kWaitLimitNs) {
-                    *abort_flag = 1;
-                    ok = 0;
-                    break;
-                }
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 1; ld_acquire_gpu(word) < target; ++spin) {
+        if (*abort_flag) return false;
+        if ((spin & 255u) == 0u) {
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2 * kWaitLimitNs) {
+                *abort_flag = 1;
+                return false;
             }
         }
     }
+    return true;
+}
+__device__ __forceinline__ bool warp_wait_arrivals(const int *word, int target, volatile int *abort_flag, int lane)
+{
+    int ok = 1;
+    if (lane == 0) ok = poll_until_at_least(word, target, abort_flag) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
@@ -273,7 +273,6 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     __shared__ __align__(8) Barriers bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ int flag_s;
     __shared__ float2 part[NG][1][128];                    // sweep 1: a group's (max, sum) of the rows on its lanes
     __shared__ __align__(16) float neg_lse2_all[256];    // -log2 of the row normaliser; -inf for padding rows
     __shared__ float t_chunk[MB][kChunkCap];              // sweep 2: per half, the key's sum over that half's rows
@@ -739,31 +738,27 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             }
             const int len2 = tc_chunk_len(im.n_r, cpu, s.omega);
             const int used2 = (im.n_r + len2 - 1) / len2;   // chunks of the unit that hold keys in sweep 2
-            if (!a.window_idx) {
-                // nothing to publish: the ticket only finds the block that clears the unit's words
-                if (threadIdx.x == 0) {
-                    int *ticket = a.sync + kSyncTickets + 2 * im.unit;
-                    if (atomicAdd(ticket, 1) == used2 - 1) {
-                        atomicExch(ticket, 0);
-                        atomicExch(ticket + 1, 0);
-                    }
+            // The block of the unit's last chunk selects for the unit (and clears the unit's words): that
+            // chunk is usually a short one, so its block is done early and the selection does not sit
+            // on the path of a block that the next wave is waiting for.  The other blocks only count
+            // themselves, without waiting for an answer.
+            int *ticket = a.sync + kSyncTickets + 2 * im.unit;
+            if (im.chunk != used2 - 1) {
+                if (a.window_idx) {
+                    __syncthreads();
+                    // release, cumulative: publishes the window scores the whole block wrote
+                    if (threadIdx.x == 0) red_release_gpu_add(ticket, 1);
+                } else if (threadIdx.x == 0) {
+                    atomicAdd(ticket, 1);
                 }
             } else {
-                // the block that completes the unit's last windows selects for the unit
                 __syncthreads();
-                if (threadIdx.x == 0) {
-                    __threadfence();   // cumulative: publishes the window scores the whole block wrote
-                    int *ticket = a.sync + kSyncTickets + 2 * im.unit;
-                    const int last = atomicAdd(ticket, 1) == used2 - 1;
-                    if (last) {
-                        atomicExch(ticket, 0);
-                        atomicExch(ticket + 1, 0);
-                        __threadfence();
-                    }
-                    flag_s = last;
+                if (threadIdx.x == 0 && poll_until_at_least(ticket, used2 - 1, &abort_s)) {
+                    atomicExch(ticket, 0);       // every other block of the unit is past its waits
+                    atomicExch(ticket + 1, 0);
                 }
                 __syncthreads();
-                if (flag_s) {
+                if (a.window_idx && !abort_s) {
                     select_topk_block<kThreads>(topk_sm, a.window_scores + (size_t)im.unit * s.kw_max, kw,
                                                 num_selected(im.n, s.alpha, s.omega, budget), s.k_max,
                                                 a.window_idx + (size_t)im.unit * s.k_max, a.kept_len + im.unit,
