@@ -12,7 +12,7 @@
 //   sweep 2  D[keys, rows] = K Q^T with the keys on the lanes: one thread owns one key and sums
 //            exp2(x_ij - lse2_i) over the rows (Eq. 2); the block then pools its windows (Eq. 3-4).
 //            The block re-reads the keys it streamed in sweep 1, now from L2.
-//   select   the block that finishes a unit's last windows runs the radix selection for that unit.
+//   select   the block of a unit's last chunk waits for the unit's other blocks and runs the selection.
 // Units are taken in waves whose keys fit L2 together.  A work item is (unit, chunk of <= 17 key
 // tiles); the persistent blocks (at most one per SM) take the items of a wave round-robin.
 //
@@ -112,9 +112,10 @@ __device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
 // Hand-over between the sweeps, per unit (all blocks are resident: cooperative launch).  A block that
 // has written the sweep-1 statistics of one chunk adds one to the unit's arrival word; a block about
 // to normalise keys of the unit waits until all of the unit's chunks have arrived.  No block waits
-// before it has finished all its sweep-1 work, so every wait ends.  The block that takes the unit's
-// last ticket in sweep 2 (every waiter of the unit is past its wait by then) clears both words for
-// the next launch.  Bounded: a warp that waits longer than two seconds gives up and sets the
+// before it has finished all its sweep-1 work, so every wait ends.  In sweep 2 every block counts
+// itself on the unit's ticket word when it is done; the block of the unit's last chunk waits for
+// that count (every waiter of the unit is past its wait by then), clears both words for the next
+// launch and selects.  Bounded: a warp that waits longer than two seconds gives up and sets the
 // block's abort flag.
 __device__ __forceinline__ int ld_acquire_gpu(const int *p)
 {
