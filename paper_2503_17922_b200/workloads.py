@@ -143,6 +143,15 @@ def batched_ragged() -> Workload:
                     TASK_AGGREGATION, 16, budget_frac=0.12, ragged=True, n_planted=-1)
 
 
+def qwen_small(l_obs: int = 16, n: int = 8192) -> Workload:
+    """The paper's second model family (section 4.1: 7 layers per group, review window 32,
+    observation window 4 or 16), with the shape of a 1.5 B model of that family: 28 layers,
+    12 query heads over 2 KV heads (G = 6, so R = 24 or 96 observation rows), head dimension 128.
+    Not one of the five benchmark configurations: a parity case for G != 4 and gamma = 7."""
+    return Workload(f"qwen-small-a{l_obs}", 6, "bf16", 1, 28, 7, 12, 2, 128, n, l_obs, 32, TASK_AGGREGATION, 16,
+                    budget_frac=0.12, n_planted=16)
+
+
 def scaled(w: Workload, **kw) -> Workload:
     """A copy of a workload with some fields replaced (smaller parity cases)."""
     return dataclasses.replace(w, **kw)

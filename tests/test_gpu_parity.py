@@ -502,6 +502,14 @@ def test_config4_needle(n, depth):
         assert len(needle) == 8 and set(needle) <= set(gpu["window_idx"][0, h].tolist())
 
 
+@pytest.mark.parametrize("l_obs", [4, 16])
+def test_second_model_family_shape(l_obs):
+    """7 layers per group, 6 query heads per KV head, review window 32, observation window 4 / 16."""
+    w = wl.qwen_small(l_obs)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=1)
+    assert len(gpu["k_out"]) == 7 and max_rel < 1e-4
+
+
 def test_config5_batched_ragged_sampled_units():
     # the leader's K of one group at full size (B = 8, n_b in [32K, 64K], packed); the oracle
     # scores a sample of units, every unit's structure and gather is checked
