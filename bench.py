@@ -68,8 +68,23 @@ def peaks() -> dict:
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops", 1590.0)),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+def score_other_floors(w, pk) -> dict:
+    """What else bounds the score kernel besides the bytes of K: the exponentials (one per row and
+    key in each of the two sweeps, on the special-function unit: 16 per clock per SM, 148 SMs,
+    1965 MHz) and the contraction (2 * R * d flops per key and sweep, against the measured bf16
+    GEMM rate).  Milliseconds per launch."""
+    keys = int(w.seqlens().sum()) * w.n_kv_heads          # (unit, key) pairs
+    rows = w.rows
+    exps = 2.0 * keys * rows
+    flops = 2.0 * 2.0 * keys * rows * w.head_dim
+    return {"ex2_floor_ms": exps / (148 * 16 * 1.965e9) * 1e3,
+            "tensor_floor_ms": flops / (pk["bf16_tflops"] * 1e12) * 1e3,
+            "hbm_floor_ms": None}
 
 
 def ncu_traffic(kernel: str):
@@ -360,6 +375,8 @@ def main() -> None:
                 "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
                 "traffic": ncu_traffic(dominant) if args.workload == "C3" else None, "algorithmic_bytes_per_launch": alg[dominant],
                 "launch_ms": dom_ms,
+                "score_kernel_floors": {**score_other_floors(w, pk),
+                                        "hbm_floor_ms": alg["score"] / (pk["hbm_gbs"] * 1e9) * 1e3},
                 "other_kernel": {"kernel": "gather_kv_kernel" if dominant == "score" else "score_windows_tc",
                                  "launch_ms": ms_gather if dominant == "score" else ms_score_select,
                                  "achieved": alg["gather" if dominant == "score" else "score"] /
