@@ -453,9 +453,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
     auto compute_stats = [&](const Item &im) {
         const int ncols = MB == 2 ? kTile : Rp;             // columns of a tile this thread reduces
         const int col0 = MB == 2 ? 0 : (L / Rp) * Rp;       // warp-uniform: Rp is a multiple of 32
-        const int gshift = ncols == 128 ? 2 : (ncols == 64 ? 1 : 0);   // log2(32-column groups per row block)
-        const int gmask = (1 << gshift) - 1;
-        const int nslot = 1 << gshift;                      // 32-column slots of an accumulator this thread reduces
+        const int nslot = ncols >> 5;                       // 32-column slots of an accumulator this thread reduces
         float m0 = -INFINITY, l0 = 0.f;
         int limit0;                                         // last key the thread's row may attend to
         {
@@ -463,7 +461,6 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             limit0 = row < s.R ? min(im.n_r + row % s.alpha, im.j_end - 1) : -1;
         }
         const uint32_t taddr = taddr_grp + col0;
-        (void)gmask;
         for (uint32_t v = it * MB; v < (it + im.n_tiles) * MB; ++v) {
             if ((int)(v % NG) != grp) continue;
             const int t = (int)(v / MB - it);

@@ -502,6 +502,15 @@ def test_config4_needle(n, depth):
         assert len(needle) == 8 and set(needle) <= set(gpu["window_idx"][0, h].tolist())
 
 
+def test_long_context_many_chunks_and_waves():
+    """131,072 keys per sequence: 148 chunks per unit, two units per wave, four waves; the selection
+    runs over 8,190 windows per unit."""
+    w = wl.scaled(wl.llama8b_full(), name="long-128K", max_seqlen=131072, n_layers=1, gamma=1, budget_frac=0.05,
+                  config_id=11)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=0)
+    assert gpu["prob"].kw_max == 8190 and max_rel < 1e-4
+
+
 @pytest.mark.parametrize("l_obs", [4, 16])
 def test_second_model_family_shape(l_obs):
     """7 layers per group, 6 query heads per KV head, review window 32, observation window 4 / 16."""
