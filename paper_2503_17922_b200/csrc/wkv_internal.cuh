@@ -95,10 +95,15 @@ __host__ __device__ inline TcPlan tc_plan(int units, int max_seqlen, int head_di
     TcPlan p;
     const long long unit_bytes = (long long)max_seqlen * head_dim * 2;
     long long upw = kTcWaveBytes / (unit_bytes > 0 ? unit_bytes : 1);
+    const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
+    // A unit needs at least ceil(max_tiles / kTcMaxChunkTiles) blocks: no more units in a wave than
+    // the SMs can take at that rate, or some blocks get two items of a wave and the others wait for
+    // them (8 sequences of up to 64 K keys: 0.70 ms with 4 units of 37 chunks per wave, 1.18 ms with 5 units of 32).
+    const int min_chunks = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
+    if (upw > kTcTargetBlocks / min_chunks) upw = kTcTargetBlocks / min_chunks;
     if (upw < 1) upw = 1;
     if (upw > units) upw = units;
     p.units_per_wave = (int)upw;
-    const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
     int a = kTcTargetBlocks / p.units_per_wave;
     const int b = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
     if (a < 1) a = 1;
