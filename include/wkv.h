@@ -34,6 +34,18 @@
  *     Q_obs element (b, hq, i, c) at q[b*q_stride_b + hq*q_stride_h + i*q_stride_t + c],
  *     i = 0..alpha-1 being positions n-alpha .. n-1 of the sequence.
  *   - Base pointers and row strides must be 16-byte aligned.
+ *   - cu_seqlens and budgets exist twice, as a HOST and as a DEVICE array.  Sizes of outputs and
+ *     of the workspace are derived from the host copies, the kernels read the device copies: the
+ *     two must hold the same values when a call is made.  The library does not compare them.  As a
+ *     guard, the kernels take no sequence to be longer and no selection to be larger than the host
+ *     copies allowed for, so a stale device copy gives wrong results, not accesses outside the
+ *     arrays sized from the host copy.
+ *   - No output may overlap an input of the same call: the gather reads K/V through the
+ *     read-only data path while other warps are already writing the compact cache, so compacting
+ *     a tensor into its own front (k_out[l] == k_layers[l]) gives undefined rows.
+ *     wkv_gather_kv and the group calls refuse identical input and output pointers of a layer
+ *     (WKV_ERR_SHAPE); partial overlaps are the caller's to avoid.  wkv_compact_kv_inplace is the
+ *     entry point for compaction inside one buffer.
  */
 #ifndef WKV_H_
 #define WKV_H_
@@ -93,6 +105,12 @@ typedef struct {
 /* ---- host-side integer helpers (Eq. 3 and the budget sentence after Eq. 4) ---- */
 int32_t wkv_num_windows(int32_t n, int32_t alpha, int32_t omega);                   /* K_w */
 int32_t wkv_num_selected(int32_t n, int32_t alpha, int32_t omega, int32_t budget);  /* k   */
+/* Rows of one unit's compact cache and, through *k_out (may be NULL), the number k of selected
+ * windows, for a sequence of n tokens: min(k*omega, n - alpha) + min(alpha, n).  This is the
+ * capacity to provide; a unit keeps (omega - size of the last window) rows fewer when k < K_w and
+ * the short last window of the sequence is among the selected ones (kept_len reports the exact
+ * count).  Returns -1 for negative n / budget or alpha, omega < 1. */
+int32_t wkv_keep_len(int32_t n, int32_t alpha, int32_t omega, int32_t budget, int32_t *k_out);
 /* Leading sizes of the output arrays for a whole batch: */
 int32_t wkv_kw_max(const wkv_shape *s);   /* max_b K_w,b, at least 1 */
 int32_t wkv_k_max(const wkv_shape *s);    /* max_b k_b,   at least 1 */
@@ -116,6 +134,14 @@ int wkv_group_budgets(int32_t n_layers, int32_t gamma, int64_t b_total, int32_t 
 /* Bytes of DEVICE scratch that wkv_score_windows / wkv_compress_group need for this
  * shape (256-byte aligned base expected).  Returns 0 for an invalid shape. */
 size_t wkv_workspace_bytes(const wkv_shape *s);
+
+/* Byte offsets, inside the workspace of this shape, of the two words through which the blocks of a
+ * launch synchronise on `unit` (a ticket count and a count of arrived statistics chunks; both are
+ * zero between launches).  Diagnostic helper (no counterpart in the paper): lets a test or a
+ * debugger inspect or disturb the hand-over without knowing the workspace layout.  Either output
+ * may be NULL.  The status word is always at byte 0. */
+int wkv_workspace_sync_words(const wkv_shape *s, int32_t unit, size_t *ticket_byte_offset,
+                             size_t *arrival_byte_offset);
 
 /*
  * Eq. 1-4 for the group's leader layer.
@@ -151,7 +177,13 @@ int wkv_score_windows(const wkv_shape *s, const void *q_obs, const void *k_leade
  *   - The first call on each device looks up the area's device address (with that device current);
  *     make that first call outside any stream capture.
  *   - All calls on a device share the one area: two calls whose kernels may overlap on the GPU
- *     (different streams, no dependency) race on it.  Calls on one stream are safe.
+ *     (different streams, no dependency) race on it.  Every call first clears the status and
+ *     synchronisation words at the head of the area, so an overlapping call does more than
+ *     corrupt scores: it wipes the arrival counts of the kernel already running, whose blocks
+ *     then sit in their bounded waits for one to two seconds and end with status bit 0 set (in
+ *     either call); the scores of both calls are invalid.  Calls on one stream are safe.
+ *   - The looked-up address belongs to the device's primary context; after cudaDeviceReset() in
+ *     this process the entry point must not be used again.
  *   - device_status  DEVICE out or NULL: receives 0, or the error bits a kernel set
  *     (1 = a bounded wait inside a kernel expired and the scores are invalid).
  * Other arguments and results exactly as wkv_score_windows.

@@ -22,7 +22,7 @@ WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05 = 0, 1, 2
 WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
-    "wkv_num_windows", "wkv_num_selected", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
+    "wkv_num_windows", "wkv_num_selected", "wkv_keep_len", "wkv_workspace_sync_words", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
     "wkv_select_leader_windows", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
     L.wkv_num_windows.argtypes = [i32, i32, i32]
     L.wkv_num_selected.restype = i32
     L.wkv_num_selected.argtypes = [i32, i32, i32, i32]
+    L.wkv_keep_len.restype = i32
+    L.wkv_keep_len.argtypes = [i32, i32, i32, i32, ctypes.POINTER(i32)]
+    L.wkv_workspace_sync_words.restype = ctypes.c_int
+    L.wkv_workspace_sync_words.argtypes = [sp, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
     for name in ("wkv_kw_max", "wkv_k_max", "wkv_keep_max"):
         getattr(L, name).restype = i32
         getattr(L, name).argtypes = [sp]
@@ -434,6 +438,21 @@ def wkv_compress_group_host(prob: Problem, q_obs_host, k_layers_host, v_layers_h
         _ptr_array(v_layers_dev), _ptr_array(k_out_dev), _ptr_array(v_out_dev), _ptr(window_idx_dev),
         _ptr(kept_len_dev), keep_capacity, _ptr(workspace), workspace.numel(), _stream(stream)),
         "wkv_compress_group_host")
+
+
+def wkv_keep_len(n: int, alpha: int, omega: int, budget: int):
+    """(row capacity of one unit's compact cache, k) for a sequence of n tokens."""
+    k = ctypes.c_int32(0)
+    rows = lib().wkv_keep_len(n, alpha, omega, budget, ctypes.byref(k))
+    return int(rows), int(k.value)
+
+
+def workspace_sync_words(prob: "Problem", unit: int):
+    """Byte offsets (ticket word, arrival word) of a unit's synchronisation words in the workspace."""
+    t, a = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib().wkv_workspace_sync_words(ctypes.byref(prob.shape), unit, ctypes.byref(t), ctypes.byref(a)),
+           "wkv_workspace_sync_words")
+    return int(t.value), int(a.value)
 
 
 def device_status(workspace) -> int:

@@ -54,7 +54,7 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
     const int n = si.n;
     const int n_r = n > s.alpha ? n - s.alpha : 0;
     const int kw = num_windows(n, s.alpha, s.omega);
-    const int k = num_selected(n, s.alpha, s.omega, si.budget);
+    const int k = num_selected_capped(n, s.alpha, s.omega, si.budget, s.k_max);
     const int *idx = prm.window_idx + (size_t)unit * s.k_max;
 
     // rows of the unit: the selected windows (only the last window of the sequence can be short,
@@ -99,6 +99,9 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
             dst_row0 = review_rows + o;
         }
         if (n_rows <= 0) continue;
+        // dense output: a unit owns keep_capacity rows (cannot trigger while the device copies of
+        // cu_seqlens / budgets equal the host copies the capacity was checked against)
+        if (!prm.cu_out && dst_row0 + n_rows > prm.keep_capacity) continue;
         const int4 *sp = src + src_row0 * src_row_vecs;
         int4 *dp = dst + dst_row0 * dst_row_vecs;
         const int n_vec = n_rows * vpr;

@@ -7,6 +7,8 @@
 // Summation orders are fixed, so results are bit-identical from run to run.
 #include "wkv_internal.cuh"
 
+#include <mutex>
+
 #include <math.h>
 
 namespace wkv {
@@ -265,6 +267,20 @@ score_pool_simt(KShape s, const T *__restrict__ q, const T *__restrict__ k,
 
 }  // namespace
 
+// The opt-in to more than 48 KB of dynamic shared memory is a property of (kernel, device): it is
+// raised once per device and kernel to the largest size asked for so far, not on every launch.
+static cudaError_t allow_dynamic_smem(const void *fn, int dev, int slot, size_t bytes)
+{
+    static std::mutex mu;
+    static size_t allowed[kMaxDevices][4] = {};
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (bytes <= allowed[dev][slot]) return cudaSuccess;
+    const cudaError_t err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (err == cudaSuccess) allowed[dev][slot] = bytes;
+    return err;
+}
+
 static int simt_chunk_keys(const KShape &ks)
 {
     int per = 512 / ks.omega;
@@ -287,14 +303,14 @@ cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const 
     const size_t smem2 = smem1 + sizeof(float) * ((size_t)r_pad + 16 * kKT +
                                                   (size_t)((chunk_keys + kKT - 1) / kKT) * kKT);
     dim3 g1(ws.n_stat_chunks, units), g2(n_score_chunks, units);
-    cudaError_t err;
-#define WKV_LAUNCH_SIMT(T)                                                                          \
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+#define WKV_LAUNCH_SIMT(T, SLOT)                                                                    \
     do {                                                                                            \
-        err = cudaFuncSetAttribute(score_stats_simt<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                   (int)smem1);                                                     \
+        err = allow_dynamic_smem(reinterpret_cast<const void *>(score_stats_simt<T>), dev, SLOT, smem1);     \
         if (err != cudaSuccess) return err;                                                         \
-        err = cudaFuncSetAttribute(score_pool_simt<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
-                                   (int)smem2);                                                     \
+        err = allow_dynamic_smem(reinterpret_cast<const void *>(score_pool_simt<T>), dev, SLOT + 1, smem2);  \
         if (err != cudaSuccess) return err;                                                         \
         if (!lse_obs)                                                                               \
             score_stats_simt<T><<<g1, kThreads, smem1, stream>>>(ks, (const T *)q, (const T *)k, stats, \
@@ -304,9 +320,9 @@ cudaError_t launch_score_simt(const KShape &ks, int dtype, const void *q, const 
                                                             ws.n_stat_chunks, r_pad, chunk_keys);   \
     } while (0)
     if (dtype == WKV_F32)
-        WKV_LAUNCH_SIMT(float);
+        WKV_LAUNCH_SIMT(float, 0);
     else
-        WKV_LAUNCH_SIMT(__nv_bfloat16);
+        WKV_LAUNCH_SIMT(__nv_bfloat16, 2);
 #undef WKV_LAUNCH_SIMT
     count_launches(lse_obs ? 1 : 2);
     return cudaGetLastError();

@@ -18,7 +18,6 @@ namespace {
 // handle for cudaGetSymbolAddress(); the device address is looked up once per device below.
 static __device__ __align__(256) unsigned char g_static_scratch[WKV_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 void *g_scratch_addr[kMaxDevices] = {};
 
@@ -64,10 +63,11 @@ extern "C" int wkv_score_windows_static(const wkv_shape *s, const void *q_obs, c
         return WKV_ERR_NULL;
     }
     const Workspace ws = plan_workspace(ks);
-    if (ws.total > (size_t)WKV_STATIC_SCRATCH_BYTES) {
+    // window_scores is the caller's here, so the part of the workspace that would hold them is not needed
+    if (ws.scores_off > (size_t)WKV_STATIC_SCRATCH_BYTES) {
         set_error_detail("this shape needs %zu bytes of scratch, the built-in area holds %zu: "
                          "use wkv_score_windows with a caller-provided workspace",
-                         ws.total, (size_t)WKV_STATIC_SCRATCH_BYTES);
+                         ws.scores_off, (size_t)WKV_STATIC_SCRATCH_BYTES);
         return WKV_ERR_LIMIT;
     }
     void *scratch = nullptr;

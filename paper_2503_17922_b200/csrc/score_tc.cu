@@ -49,7 +49,6 @@ __host__ __device__ constexpr int block_threads(int mb) { return 64 + groups_for
 constexpr int kTile = kTcTileKeys;                       // keys per tile
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
 constexpr int kChunkCap = kTcMaxChunkTiles * kTile + kTcMaxWindow;   // token scores a block may hold
-constexpr int kSyncTickets = 16;                         // per unit u: sync[16 + 2u] ticket, sync[17 + 2u] sweep-1 arrivals
 
 struct TcArgs {
     KShape s;
@@ -318,7 +317,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.h = unit % s.hkv;
         if (s.cu) {
             const int lo = s.cu[im.b];
-            im.n = s.cu[im.b + 1] - lo;
+            im.n = min(max(s.cu[im.b + 1] - lo, 0), s.n_cap);
             im.off = lo;
         } else {
             im.n = s.max_seqlen;
@@ -758,7 +757,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 __syncthreads();
                 if (a.window_idx && !abort_s) {
                     select_topk_block<kThreads>(topk_sm, a.window_scores + (size_t)im.unit * s.kw_max, kw,
-                                                num_selected(im.n, s.alpha, s.omega, budget), s.k_max,
+                                                num_selected_capped(im.n, s.alpha, s.omega, budget, s.k_max), s.k_max,
                                                 a.window_idx + (size_t)im.unit * s.k_max, a.kept_len + im.unit,
                                                 im.n, s.alpha, s.omega);
                 }
@@ -861,29 +860,37 @@ bool make_key_tensor_map(const KShape &ks, const void *k, CUtensorMap *tmap, int
     return true;
 }
 
-// what the launcher needs to know about the current device and its kernels, looked up once
+// What the launcher needs to know about a device and its copy of the kernels, looked up on the first
+// use of that device: kernel attributes (the shared-memory opt-in) belong to a device, so a process
+// that drives several GPUs sets them on each.
 struct DeviceInfo {
+    bool known = false;
     int cc_major = -1;
     int sm_count = 0;
     int cooperative = 0;
     int blocks_per_sm[2] = {-1, -1};   // resident blocks of each instantiation at its largest footprint
 };
-DeviceInfo &device_info()
+std::mutex g_device_mutex;
+DeviceInfo g_device_info[kMaxDevices];
+// the current device's entry (callers hold no lock: entries are only ever filled in, under the mutex)
+DeviceInfo *device_info()
 {
-    static DeviceInfo info;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return;
-        }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    DeviceInfo &info = g_device_info[dev];
+    if (!info.known) {
         int v = 0;
         if (cudaDeviceGetAttribute(&v, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess) info.cc_major = v;
         if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) info.sm_count = v;
         if (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess) info.cooperative = v;
-    });
-    return info;
+        (void)cudaGetLastError();
+        info.known = true;
+    }
+    return &info;
 }
 
 size_t tc_smem_bytes(int kblocks, int mb)
@@ -895,9 +902,9 @@ size_t tc_smem_bytes(int kblocks, int mb)
 
 bool score_tc_supported(const KShape &ks, int dtype)
 {
-    const DeviceInfo &di = device_info();
-    return dtype == WKV_BF16 && (ks.d == 64 || ks.d == 128) && ks.R <= 256 && ks.omega <= kTcMaxWindow &&
-           di.cc_major == 10 && di.cooperative && di.sm_count > 0;
+    const DeviceInfo *di = device_info();
+    return di && dtype == WKV_BF16 && (ks.d == 64 || ks.d == 128) && ks.R <= 256 && ks.omega <= kTcMaxWindow &&
+           di->cc_major == 10 && di->cooperative && di->sm_count > 0;
 }
 
 int launch_score_tc(const KShape &ks, const void *q, const void *k, float *window_scores, float *token_scores,
@@ -907,7 +914,12 @@ int launch_score_tc(const KShape &ks, const void *q, const void *k, float *windo
     alignas(64) CUtensorMap tmap;
     int slot[3] = {1, 2, 3};
     if (!make_key_tensor_map(ks, k, &tmap, slot)) return WKV_ERR_UNSUPPORTED;
-    DeviceInfo &di = device_info();
+    DeviceInfo *dip = device_info();
+    if (!dip) {
+        set_error_detail("no current CUDA device, or its ordinal is beyond %d", kMaxDevices - 1);
+        return WKV_ERR_CUDA;
+    }
+    DeviceInfo &di = *dip;
 
     TcArgs a;
     a.s = ks;
@@ -937,8 +949,9 @@ int launch_score_tc(const KShape &ks, const void *q, const void *k, float *windo
     const void *fn = mb == 1 ? reinterpret_cast<const void *>(score_windows_tc<1>)
                              : reinterpret_cast<const void *>(score_windows_tc<2>);
     cudaError_t err = cudaSuccess;
+    std::unique_lock<std::mutex> setup_lock(g_device_mutex);
     if (di.blocks_per_sm[mb - 1] < 0) {
-        // once per instantiation: allow its largest shared-memory request (head_dim 128) and ask how
+        // once per device and instantiation: allow its largest shared-memory request (head_dim 128) and ask how
         // many of its blocks an SM holds at that size
         const size_t smem_max = tc_smem_bytes(2, mb);
         err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
@@ -957,6 +970,7 @@ int launch_score_tc(const KShape &ks, const void *q, const void *k, float *windo
             di.blocks_per_sm[mb - 1] = occ;
         }
     }
+    setup_lock.unlock();
     // persistent blocks, one per SM at most; every block of a cooperative launch is resident, which
     // the hand-over of the statistics between the sweeps relies on
     int grid = plan.units_per_wave * plan.chunks_per_unit;

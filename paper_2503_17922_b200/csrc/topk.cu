@@ -15,7 +15,7 @@ select_topk_kernel(KShape s, const float *__restrict__ window_scores, int *__res
     const int b = unit / s.hkv;
     const SeqInfo si = seq_info(s, b);
     const int kw = num_windows(si.n, s.alpha, s.omega);
-    const int k = num_selected(si.n, s.alpha, s.omega, si.budget);
+    const int k = num_selected_capped(si.n, s.alpha, s.omega, si.budget, s.k_max);
     select_topk_block<kThreads>(sm, window_scores + (size_t)unit * s.kw_max, kw, k, s.k_max,
                                 window_idx + (size_t)unit * s.k_max, kept_len + unit, si.n, s.alpha, s.omega);
 }

@@ -153,6 +153,10 @@ int resolve(const wkv_shape *s, KShape &ks)
     ks.k_max = k_max;
     ks.nr_max = s->max_seqlen - s->l_obs > 1 ? s->max_seqlen - s->l_obs : 1;
     (void)nr_max;
+    {
+        const long long cap = (long long)s->l_obs + (long long)kw_max * s->window;
+        ks.n_cap = cap < s->max_seqlen ? (int)cap : s->max_seqlen;
+    }
     ks.cu = s->cu_seqlens_dev;
     ks.budgets = s->budgets_dev;
     ks.sb = s->stride_b;
@@ -260,6 +264,11 @@ static int fill_table(int n_layers, const void *const *k_layers, const void *con
                 set_error_detail("layer %d: tensor pointer not 16-byte aligned", l);
                 return WKV_ERR_ALIGN;
             }
+            if (src[t] == dst[t]) {
+                set_error_detail("layer %d: the compact cache must not be the input tensor itself "
+                                 "(wkv_compact_kv_inplace compacts inside one buffer)", l);
+                return WKV_ERR_SHAPE;
+            }
             tab.src[n_tensors] = src[t];
             tab.dst[n_tensors] = dst[t];
             ++n_tensors;
@@ -291,6 +300,37 @@ int32_t wkv_num_windows(int32_t n, int32_t alpha, int32_t omega) { return num_wi
 int32_t wkv_num_selected(int32_t n, int32_t alpha, int32_t omega, int32_t budget)
 {
     return num_selected(n, alpha, omega, budget);
+}
+
+int32_t wkv_keep_len(int32_t n, int32_t alpha, int32_t omega, int32_t budget, int32_t *k_out)
+{
+    if (n < 0 || alpha < 1 || omega < 1 || budget < 0) {
+        if (k_out) *k_out = 0;
+        return -1;
+    }
+    const int k = num_selected(n, alpha, omega, budget);
+    if (k_out) *k_out = k;
+    const int n_r = n > alpha ? n - alpha : 0;
+    const long long rows = (long long)k * omega;
+    // all windows selected: the short last window is among them and the cache is the whole sequence
+    return (int32_t)((rows < n_r ? rows : n_r) + (n < alpha ? n : alpha));
+}
+
+int wkv_workspace_sync_words(const wkv_shape *s, int32_t unit, size_t *ticket_byte_offset,
+                             size_t *arrival_byte_offset)
+{
+    KShape ks;
+    const int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (unit < 0 || unit >= ks.batch * ks.hkv) {
+        set_error_detail("unit %d outside 0..%d", unit, ks.batch * ks.hkv - 1);
+        return WKV_ERR_SHAPE;
+    }
+    const Workspace ws = plan_workspace(ks);
+    const size_t ticket = ws.sync_off + sizeof(int) * ((size_t)kSyncTickets + 2 * (size_t)unit);
+    if (ticket_byte_offset) *ticket_byte_offset = ticket;
+    if (arrival_byte_offset) *arrival_byte_offset = ticket + sizeof(int);
+    return WKV_OK;
 }
 
 int32_t wkv_kw_max(const wkv_shape *s)
@@ -537,6 +577,32 @@ int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers, const void *q_
         !k_out_layers_dev || !v_out_layers_dev || !window_idx_dev || !kept_len_dev) {
         set_error_detail("a host or staging pointer is NULL");
         return WKV_ERR_NULL;
+    }
+    // the byte counts are the caller's: they must cover what the shape says the kernels will touch,
+    // and the output count must be exactly one dense compact cache
+    {
+        const size_t eb = (size_t)elem_bytes(s->dtype);
+        const size_t rows = ks.cu ? (size_t)ks.total_rows : (size_t)ks.max_seqlen;
+        const size_t kv_extent = ((rows - 1) * (size_t)ks.st + (size_t)(ks.batch - 1) * (size_t)ks.sb +
+                                  (size_t)(ks.hkv - 1) * (size_t)ks.sh + (size_t)ks.d) * eb;
+        const size_t q_extent = ((size_t)(ks.batch - 1) * (size_t)ks.qsb + (size_t)(ks.hq - 1) * (size_t)ks.qsh +
+                                 (size_t)(ks.alpha - 1) * (size_t)ks.qst + (size_t)ks.d) * eb;
+        if (bytes_per_layer < kv_extent || q_bytes < q_extent) {
+            set_error_detail("host buffers smaller than the shape: bytes_per_layer %zu (needs %zu), q_bytes %zu "
+                             "(needs %zu)", bytes_per_layer, kv_extent, q_bytes, q_extent);
+            return WKV_ERR_SHAPE;
+        }
+        if (keep_capacity < keep_max_of(s)) {
+            set_error_detail("keep_capacity %d smaller than the %d rows a unit may keep", keep_capacity,
+                             keep_max_of(s));
+            return WKV_ERR_SHAPE;
+        }
+        const size_t out_exact = (size_t)ks.batch * ks.hkv * (size_t)keep_capacity * ks.d * eb;
+        if (out_bytes_per_layer != out_exact) {
+            set_error_detail("out_bytes_per_layer %zu is not one dense compact cache [B, H_kv, keep_capacity, d] "
+                             "= %zu bytes", out_bytes_per_layer, out_exact);
+            return WKV_ERR_SHAPE;
+        }
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     st = check_cuda(cudaMemcpyAsync(q_obs_dev, q_obs_host, q_bytes, cudaMemcpyHostToDevice, stream), "copy of q_obs");

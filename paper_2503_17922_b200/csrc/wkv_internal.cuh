@@ -20,6 +20,10 @@ struct KShape {
     int total_rows;            // sum of the sequence lengths (rows of the packed layout)
     int G, R;                  // query heads per KV head; observation rows per unit = G*alpha
     int kw_max, k_max, nr_max; // leading sizes of window_scores / window_idx / token_scores
+    int n_cap;                 // no sequence is taken to be longer than this on the device:
+                               // min(max_seqlen, alpha + kw_max * omega), so that a device copy of
+                               // cu_seqlens that disagrees with the host copy cannot lead a kernel
+                               // past the arrays that were sized from the host copy
     const int *cu;             // device cu_seqlens or nullptr
     const int *budgets;        // device budgets or nullptr
     long long sb, sh, st;      // K/V element strides
@@ -39,6 +43,12 @@ __host__ __device__ inline int num_selected(int n, int alpha, int omega, int bud
     int k = budget > alpha ? (budget - alpha) / omega : 0;
     return k < kw ? k : kw;
 }
+// the same, never beyond the leading size of window_idx (device side: budgets_dev is not trusted further)
+__host__ __device__ inline int num_selected_capped(int n, int alpha, int omega, int budget, int k_max)
+{
+    const int k = num_selected(n, alpha, omega, budget);
+    return k < k_max ? k : k_max;
+}
 
 struct SeqInfo {
     int n;          // context length
@@ -52,6 +62,7 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
     if (s.cu) {
         int lo = s.cu[b];
         r.n = s.cu[b + 1] - lo;
+        r.n = r.n < 0 ? 0 : (r.n > s.n_cap ? s.n_cap : r.n);
         r.off = lo;
     } else {
         r.n = s.max_seqlen;
@@ -72,6 +83,13 @@ struct Workspace {
     int n_stat_chunks;
     int r_pad;
 };
+
+// words of the synchronisation area before the per-unit words: unit u owns sync[kSyncTickets + 2u]
+// (ticket) and sync[kSyncTickets + 2u + 1] (arrivals of the statistics sweep)
+constexpr int kSyncTickets = 16;
+
+// per-device host state (kernel attributes, device properties) is kept for this many device ordinals
+constexpr int kMaxDevices = 64;
 
 constexpr int kStatChunk = 512;   // keys per partial-statistics chunk of the CUDA-core kernels
 

@@ -103,6 +103,69 @@ def test_null_workspace_alignment_and_limits(L):
     assert L.wkv_launch_count() == 0
 
 
+def test_keep_len_matches_the_oracle_formulas(L):
+    k = ctypes.c_int32(-5)
+    for n in (1, 7, 8, 9, 17, 100, 1024, 1027, 32768):
+        for a in (1, 8, 32):
+            for w in (1, 3, 8, 16, 32):
+                for b in (0, a, a + w - 1, a + w, 983, 10 ** 6):
+                    rows = L.wkv_keep_len(n, a, w, b, ctypes.byref(k))
+                    k_ref = oracle.num_selected(n, a, w, b)
+                    assert k.value == k_ref
+                    n_r = max(n - a, 0)
+                    # the largest set of k windows in rows: the k first ones (all full unless k == K_w)
+                    assert rows == min(k_ref * w, n_r) + min(a, n)
+                    assert rows == oracle.keep_max([n], [b], a, w) or k_ref == oracle.num_windows(n, a, w)
+                    assert rows <= n and (b < a or rows <= max(b, min(a, n)))
+    assert L.wkv_keep_len(100, 8, 8, 64, None) == 64      # k = 7 windows of 8 + 8 observation rows
+    assert L.wkv_keep_len(-1, 8, 8, 64, None) == -1 and L.wkv_keep_len(10, 0, 8, 64, None) == -1
+
+
+def test_sync_word_helper(L):
+    s = _shape()
+    t, a = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    need = L.wkv_workspace_bytes(ctypes.byref(s))
+    seen = set()
+    for unit in range(2):
+        assert L.wkv_workspace_sync_words(ctypes.byref(s), unit, ctypes.byref(t), ctypes.byref(a)) == 0
+        assert 4 <= t.value < a.value < need and t.value % 4 == 0 and a.value % 4 == 0
+        seen |= {t.value, a.value}
+    assert len(seen) == 4
+    assert L.wkv_workspace_sync_words(ctypes.byref(s), 2, ctypes.byref(t), ctypes.byref(a)) == 2
+    assert L.wkv_workspace_sync_words(ctypes.byref(s), 0, None, None) == 0
+
+
+def test_host_entry_refuses_byte_counts_that_disagree_with_the_shape(L):
+    """wkv_compress_group_host copies caller-sized byte ranges: sizes that do not cover the tensors
+    of the shape, or an output size that is not exactly one dense compact cache, are refused on the
+    host before any copy is enqueued (no GPU needed to see the refusal)."""
+    s = _shape()
+    ptrs = (ctypes.c_void_p * 4)(*([0x1000] * 4))
+    kv_bytes = 2 * 1024 * 64 * 2
+    q_bytes = 4 * 8 * 64 * 2
+    cap = L.wkv_keep_max(ctypes.byref(s))
+    out_bytes = 2 * cap * 64 * 2
+    need = L.wkv_workspace_bytes(ctypes.byref(s))
+
+    def call(qb=q_bytes, kb=kv_bytes, ob=out_bytes, capacity=cap):
+        return L.wkv_compress_group_host(ctypes.byref(s), 2, 0x1000, qb, ptrs, ptrs, kb, ptrs, ptrs, ob, 0x1000, 0x1000,
+                                         0x1000, ptrs, ptrs, ptrs, ptrs, 0x1000, 0x1000, capacity, 0x1000, need, None)
+    assert call(kb=kv_bytes - 2) == 2 and b"bytes_per_layer" in L.wkv_last_error_detail()
+    assert call(qb=q_bytes - 2) == 2
+    assert call(ob=out_bytes - 2) == 2 and b"out_bytes_per_layer" in L.wkv_last_error_detail()
+    assert call(ob=out_bytes + 128) == 2
+    assert call(capacity=cap - 1, ob=2 * (cap - 1) * 64 * 2) == 2
+    assert L.wkv_launch_count() == 0
+
+
+def test_gather_refuses_a_cache_that_is_its_own_input(L):
+    s = _shape()
+    a = (ctypes.c_void_p * 2)(0x1000, 0x2000)
+    b = (ctypes.c_void_p * 2)(0x3000, 0x2000)      # layer 1: output == input
+    assert L.wkv_gather_kv(ctypes.byref(s), 2, a, None, 0x100, b, None, None, 128, None) == 2
+    assert b"must not be the input" in L.wkv_last_error_detail()
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libwkv.so")

@@ -259,6 +259,54 @@ def test_gather_spot_checks_and_budget_invariants(ragged):
             assert set(planted) <= set(sel), "planted windows must be retained"
 
 
+@pytest.mark.parametrize("ragged", [False, True])
+def test_gather_into_the_packed_output_layout(ragged):
+    """The packed compact cache [T_out, H_kv, d]: sequence b starts at row cu_seqlens_out[b], its rows
+    are token-major with the KV heads interleaved.  Every output element is located here by index
+    arithmetic written independently of the oracle's gather loop, on given (not selected) indices
+    that differ per head and include the ragged last window; slack rows between sequences and rows
+    behind a unit's kept length must keep the fill."""
+    w = _small_group(ragged=ragged)
+    grp = wl.make_group(w, 0)
+    seqlens, cu = grp["seqlens"], grp["cu_seqlens"]
+    H, d = w.n_kv_heads, w.head_dim
+    ks = [oracle.num_selected(int(n), w.l_obs, w.window, int(b)) for n, b in zip(seqlens, grp["budgets"])]
+    k_max = max(ks)
+    idx = np.full((w.batch, H, k_max), -1, dtype=np.int32)
+    for b in range(w.batch):
+        kw = oracle.num_windows(int(seqlens[b]), w.l_obs, w.window)
+        for h in range(H):
+            # head 0: every other window and the (short) last one; head 1: the first k windows
+            cand = np.unique(np.concatenate([np.arange(h, kw, 2)[: ks[b] - 1], [kw - 1]]))[: ks[b]] if h == 0 \
+                else np.arange(ks[b])
+            assert len(cand) == ks[b]
+            idx[b, h, : ks[b]] = cand
+    slack = [3, 0, 5][: w.batch]                       # unused rows behind each sequence's share
+    cu_out = np.zeros(w.batch + 1, dtype=np.int32)
+    for b in range(w.batch):
+        cu_out[b + 1] = cu_out[b] + ks[b] * w.window + w.l_obs + slack[b]
+    FILL = 0x5A5A
+    src = grp["v_layers"][1]
+    out = oracle.gather_layer(src, idx, n_kv_heads=H, l_obs=w.l_obs, window=w.window, max_seqlen=w.max_seqlen,
+                              budgets=grp["budgets"], keep_max=0, cu_seqlens=cu, cu_seqlens_out=cu_out, fill=FILL)
+    assert out.shape == (int(cu_out[-1]), H, d)
+    flat = out.reshape(-1)                              # element (row, h, c) at (row * H + h) * d + c
+    written = np.zeros(out.shape[:2], dtype=bool)
+    for b in range(w.batch):
+        n = int(seqlens[b]); n_r = n - w.l_obs
+        for h in range(H):
+            rows = np.concatenate([np.arange(i * w.window, min((i + 1) * w.window, n_r)) for i in idx[b, h, : ks[b]]]
+                                  + [np.arange(n_r, n)])
+            src_u = src[cu[b]:cu[b + 1], h] if ragged else src[b, h]
+            for r, j in enumerate(rows):
+                base = ((int(cu_out[b]) + r) * H + h) * d
+                np.testing.assert_array_equal(flat[base: base + d], src_u[j])
+                written[int(cu_out[b]) + r, h] = True
+            # head 0 holds the short last window, head 1 does not: the kept lengths differ
+            assert len(rows) == ks[b] * w.window + w.l_obs - (w.window - (n_r - (oracle.num_windows(n, w.l_obs, w.window) - 1) * w.window) if h == 0 else 0)
+    assert (out[~written] == FILL).all() and (~written).sum() > 0
+
+
 def test_budget_above_context_is_identity_copy():
     w = wl.scaled(_small_group(), budget_frac=None, budget_tokens=10 ** 6)
     grp = wl.make_group(w, 0)
