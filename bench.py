@@ -73,73 +73,121 @@ def peaks() -> dict:
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
-def score_other_floors(w, pk) -> dict:
-    """What else bounds the score kernel besides the bytes of K: the exponentials (one per row and
-    key in each of the two sweeps, on the special-function unit: 16 per clock per SM, 148 SMs,
-    1965 MHz) and the contraction (2 * R * d flops per key and sweep, against the measured bf16
-    GEMM rate).  Milliseconds per launch."""
+def score_other_floors(w, pk, ex2_per_s: float) -> dict:
+    """What else bounds the score stage besides the bytes of K: the exponentials (one per row and
+    key in each of the two sweeps, at the rate the ex2 probe measured on this GPU in this run) and
+    the contraction (2 * R * d flops per key and sweep, against the measured bf16 GEMM rate).
+    Milliseconds per launch."""
     keys = int(w.seqlens().sum()) * w.n_kv_heads          # (unit, key) pairs
     rows = w.rows
     exps = 2.0 * keys * rows
     flops = 2.0 * 2.0 * keys * rows * w.head_dim
-    return {"ex2_floor_ms": exps / (148 * 16 * 1.965e9) * 1e3,
-            "tensor_floor_ms": flops / (pk["bf16_tflops"] * 1e12) * 1e3,
-            "hbm_floor_ms": None}
+    return {"ex2_floor_ms": exps / ex2_per_s * 1e3, "ex2_per_s_measured": ex2_per_s,
+            "ex2_per_clk_per_sm_at_1965mhz": ex2_per_s / (148 * 1.965e9),
+            "tensor_floor_ms": flops / (pk["bf16_tflops"] * 1e12) * 1e3}
 
 
-def ncu_traffic(kernel: str):
-    """DRAM bytes per launch of the kernel from the committed ncu capture (config 3 only), or None."""
+def kernel_source_hash() -> str:
+    """Fingerprint of the kernel sources: the ncu traffic figures are only quoted while it is unchanged."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_17922_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(name.encode())
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of the kernel from the committed ncu capture, or None when there is no
+    capture of this kernel on this workload or the kernel sources have changed since it was taken."""
     p = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
-    if os.path.exists(p):
-        for line in open(p):
-            f = line.split()
-            if len(f) == 2 and f[0] == kernel:
-                return int(f[1])
-    return None
+    if not os.path.exists(p):
+        return None
+    found, current = None, False
+    for line in open(p):
+        f = line.split()
+        if len(f) == 2 and f[0] == "sources":
+            current = f[1] == kernel_source_hash()
+        if len(f) == 3 and f[0] == kernel and f[1] == workload:
+            found = int(f[2])
+    return found if current else None
 
 
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Read-only sampling of the current GPU's clocks with nvidia-smi (selected by UUID, so that
+    CUDA_VISIBLE_DEVICES cannot point it at another GPU), written to a file so that no sample is lost
+    when the sampler is stopped.  It runs for the whole process; `mark()` notes the start and end of
+    the timed region, and the summary says how many samples fell inside it."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index = index
-        self.proc = None
+    def __init__(self, uuid: str, period_ms: int = 20):
+        import tempfile
+        self.uuid, self.period_ms = uuid, period_ms
+        self.proc, self.marks = None, []
+        self.path = os.path.join(tempfile.gettempdir(), f"wkv_clocks_{os.getpid()}.csv")
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "20"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.uuid}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", str(self.period_ms),
+                                          "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
+    def mark(self):
+        self.marks.append(time.time())
+
     def stop(self) -> dict:
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(2.5 * self.period_ms / 1e3)
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[1]), float(f[2]), f[4:8]))
+                except ValueError:
+                    continue
+            os.remove(self.path)
+        except OSError:
+            pass
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1]))
-                mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+        def summary(sel):
+            reasons = set()
+            for _, _, _, flags in sel:
+                for nm, val in zip(names, flags):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+            return {"sm_mhz": statistics.median(r[1] for r in sel) if sel else None,
+                    "sm_max_mhz": max((r[2] for r in sel), default=None), "samples": len(sel),
+                    "reasons": sorted(reasons)}
+        inside = [r for r in rows if len(self.marks) >= 2 and self.marks[0] <= r[0] <= self.marks[1]]
+        out = summary(inside)
+        if len(inside) < 3:
+            # the timed region is shorter than a few sampling periods: report what the GPU did while this
+            # process had it under load (warm-up, timed region and the stage timings that follow)
+            out = summary(rows)
+            out["window"] = "whole process (timed region shorter than the sampling period)"
+        else:
+            out["window"] = "timed region"
+        if not rows:
+            out["reasons"] = ["no sample could be read from nvidia-smi"]
+        return out
 
 
 def time_oracle_groups(w, groups, min_seconds: float, max_groups: int):
@@ -200,7 +248,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=40)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
-    ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05"])
+    ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05", "unfused"])
     ap.add_argument("--groups", type=int, default=0, help="distinct groups kept on the device (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -214,16 +262,28 @@ def main() -> None:
     import torch
     from paper_2503_17922_b200 import binding, replicas
 
-    # replicas only: every rank runs the whole path on its own copy of the workload (no exchange step)
+    # replicas only: every rank runs the whole path on its own copy of the workload (no exchange step).
+    # Asked for N > 1 as a plain command (no launcher environment), the benchmark starts its N ranks itself.
+    if args.gpus > 1 and not replicas.launcher_present():
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus}: only {torch.cuda.device_count()} CUDA devices are visible")
+        sys.exit(replicas.relaunch_under_launcher(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
     rank, world, local = replicas.rank_env()
     torch.cuda.set_device(local)
     replicas.init("nccl", torch.device("cuda", local))
     binding.lib()          # fails loudly if the CUDA library is missing
+    sampler = None
+    if rank == 0:
+        uuid = str(torch.cuda.get_device_properties(local).uuid)
+        sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+        sampler.start()
 
     w = pick_workload(args.workload)
     impl = {"auto": binding.WKV_SCORE_AUTO, "simt": binding.WKV_SCORE_SIMT,
-            "tcgen05": binding.WKV_SCORE_TCGEN05}[args.score_impl]
+            "tcgen05": binding.WKV_SCORE_TCGEN05, "unfused": binding.WKV_SCORE_TCGEN05_UNFUSED}[args.score_impl]
     prob = binding.Problem.from_workload(w, score_impl=impl)
+    prob_unfused = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05_UNFUSED) \
+        if (impl == binding.WKV_SCORE_AUTO and w.dtype == "bf16") else None
     alg = algorithmic_bytes(w, prob)
     tokens = alg["tokens"]
     warmup = max(args.warmup, 3)
@@ -254,6 +314,15 @@ def main() -> None:
                                                   keep_capacity=cap, stream=stream) for d in dev_groups]
     score_calls = [binding.prepare_score_windows(prob, d["q"], d["k"][0], out["window_scores"], None, work,
                                                  stream=stream) for d in dev_groups]
+    leader_calls = [binding.prepare_select_leader_windows(prob, d["q"], d["k"][0], out["window_scores"],
+                                                          out["window_idx"], out["kept_len"], work, stream=stream)
+                    for d in dev_groups]
+    unfused_calls = None
+    if prob_unfused is not None:
+        unfused_calls = [binding.prepare_compress_group(prob_unfused, d["q"], d["k"], d["v"], out["k_out"],
+                                                        out["v_out"], out["window_scores"], out["window_idx"],
+                                                        out["kept_len"], work, keep_capacity=cap, stream=stream)
+                         for d in dev_groups]
     select_call = binding.prepare_select_topk_windows(prob, out["window_scores"], out["window_idx"],
                                                       out["kept_len"], stream=stream)
     gather_calls = [binding.prepare_gather_kv(prob, d["k"], d["v"], out["window_idx"], out["k_out"], out["v_out"],
@@ -272,9 +341,8 @@ def main() -> None:
                 flush.fill_(i & 0xFF)
             plans[i % n_groups].launch(stream)
         barrier()
-        sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
+        if sampler:
+            sampler.mark()
         launches0 = binding.wkv_launch_count()
         if flush is None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -295,7 +363,8 @@ def main() -> None:
             barrier()
             ms_total = sum(a.elapsed_time(b) for a, b in evs)
         launches = binding.wkv_launch_count() - launches0
-        clocks = sampler.stop() if rank == 0 else None
+        if sampler:
+            sampler.mark()
         ms_total = replicas.max_over_ranks(ms_total, "cuda")
         ms_per_step = ms_total / args.steps
         value = replicas.whole_job_rate(tokens, world, ms_per_step)
@@ -350,8 +419,19 @@ def main() -> None:
             d1.record(stream)
             stream.synchronize()
             ms_direct = d0.elapsed_time(d1) / n_direct
-        ms_fused = time_stage(group_calls)                 # score+select kernel followed by the gather kernel
-        ms_score = time_stage(score_calls)                 # the same kernel without the selection
+        ms_fused = time_stage(group_calls)                 # the group call's launch(es), graph replay
+        ms_score = time_stage(score_calls)                 # scores and pooling only
+        ms_score_select = time_stage(leader_calls)         # scores, pooling and selection in one launch, timed directly
+        ms_unfused = time_stage(unfused_calls) if unfused_calls else None   # two-launch form of the group
+        # the special-function rate of this GPU, measured: 148 x 4 blocks of 1024 threads, 8 chains each
+        probe_scratch = torch.zeros(4, dtype=torch.float32, device="cuda")
+        binding.wkv_probe_ex2_rate(probe_scratch, 592, 1024, 64, stream=stream)
+        pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pa.record(stream)
+        n_ex2 = binding.wkv_probe_ex2_rate(probe_scratch, 592, 1024, 4096, stream=stream)
+        pb.record(stream)
+        stream.synchronize()
+        ex2_per_s = n_ex2 / (pa.elapsed_time(pb) * 1e-3)
         ms_select = time_stage([select_call])              # stand-alone selection kernel (not on the fused path)
         ms_gather = time_stage(gather_calls)
         # the variant that takes Eq. 1's normalisers from the caller (no statistics sweep); the inputs of
@@ -364,23 +444,36 @@ def main() -> None:
                                                             out["kept_len"], work, keep_capacity=cap, stream=stream)
                          for d, l in zip(dev_groups, lse)]
             ms_given_lse = time_stage(lse_calls)
-    ms_score_select = max(ms_fused - ms_gather, ms_score)  # fused score+selection kernel on the group path
+    clocks = sampler.stop() if sampler else None
 
     pk = peaks()
-    dominant = "gather" if ms_gather >= ms_score_select else "score"
-    dom_ms = ms_gather if dominant == "gather" else ms_score_select
-    achieved = alg[dominant] / (dom_ms * 1e-3) / 1e9
-    kernel_name = "gather_kv_kernel" if dominant == "gather" else "score_windows_tc (both sweeps + selection)"
-    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": pk["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "peak_source": pk["source"],
-                "traffic": ncu_traffic(dominant) if args.workload == "C3" else None, "algorithmic_bytes_per_launch": alg[dominant],
-                "launch_ms": dom_ms,
-                "score_kernel_floors": {**score_other_floors(w, pk),
-                                        "hbm_floor_ms": alg["score"] / (pk["hbm_gbs"] * 1e9) * 1e3},
-                "other_kernel": {"kernel": "gather_kv_kernel" if dominant == "score" else "score_windows_tc",
-                                 "launch_ms": ms_gather if dominant == "score" else ms_score_select,
-                                 "achieved": alg["gather" if dominant == "score" else "score"] /
-                                 ((ms_gather if dominant == "score" else ms_score_select) * 1e-3) / 1e9}}
+    floors = score_other_floors(w, pk, ex2_per_s)
+    floors["hbm_floor_ms"] = alg["score"] / (pk["hbm_gbs"] * 1e9) * 1e3
+    launches_per_step = launches / args.steps
+    if launches_per_step < 1.5:
+        # the whole group is ONE launch (scores, selection and gather in the pipelined kernel): its
+        # duration is the time per step of the timed region, its bytes are the path's
+        dom_ms, dom_bytes, kernel_key = ms_per_step, alg["total"], "group_pipeline"
+        roofline = {"bound": "hbm", "kernel": "group_pipeline_tc (scores + pooling + selection + gather, one launch)",
+                    "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "peak_source": pk["source"], "traffic": ncu_traffic(kernel_key, w.name),
+                    "algorithmic_bytes_per_launch": dom_bytes, "launch_ms": dom_ms,
+                    "launch_ms_source": "timed region / launches (CUDA events on the launching stream)",
+                    "score_stage_floors": floors}
+    else:
+        dominant = "gather" if ms_gather >= ms_score_select else "score"
+        dom_ms = ms_gather if dominant == "gather" else ms_score_select
+        other = "score" if dominant == "gather" else "gather"
+        other_ms = ms_score_select if dominant == "gather" else ms_gather
+        names = {"gather": "gather_kv_kernel", "score": "score kernel (both sweeps + pooling + selection)"}
+        roofline = {"bound": "hbm", "kernel": names[dominant], "achieved": alg[dominant] / (dom_ms * 1e-3) / 1e9,
+                    "peak": pk["hbm_gbs"], "unit": "GB/s", "peak_source": pk["source"],
+                    "traffic": ncu_traffic(dominant, w.name), "algorithmic_bytes_per_launch": alg[dominant],
+                    "launch_ms": dom_ms, "launch_ms_source": "the launch alone, graph replay between CUDA events",
+                    "score_stage_floors": floors,
+                    "other_kernel": {"kernel": names[other], "launch_ms": other_ms,
+                                     "achieved": alg[other] / (other_ms * 1e-3) / 1e9}}
+    roofline["frac"] = roofline["achieved"] / pk["hbm_gbs"]
     path_frac = alg["total"] / (ms_per_step * 1e-3) / 1e9 / pk["hbm_gbs"]
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
@@ -442,8 +535,9 @@ def main() -> None:
             "gpu_launches": int(launches),
             "path_hbm_frac": path_frac,
             "path_algorithmic_bytes": alg["total"],
-            "stages_ms": {"group_graph_replay": ms_fused, "score_select_fused": ms_score_select,
-                          "score_only": ms_score, "select_standalone": ms_select, "gather": ms_gather,
+            "stages_ms": {"group_graph_replay": ms_fused, "group_two_launch_form": ms_unfused,
+                          "score_select_one_launch": ms_score_select,
+                          "score_only": ms_score, "select_standalone": ms_select, "gather_standalone": ms_gather,
                           "group_given_lse_graph_replay": ms_given_lse,
                           "group_direct_call": ms_direct},
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "clocks": clocks,

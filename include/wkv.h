@@ -74,8 +74,10 @@ typedef enum { WKV_F32 = 0, WKV_BF16 = 1 } wkv_dtype;
 typedef enum { WKV_TASK_LOCALIZATION = 0, WKV_TASK_AGGREGATION = 1 } wkv_task;
 /* which score kernel family to use: AUTO picks the tensor-core (tcgen05) kernels
  * for bf16 inputs with head_dim 64 or 128 and G*alpha <= 256, else the plain
- * CUDA-core kernels. */
-typedef enum { WKV_SCORE_AUTO = 0, WKV_SCORE_SIMT = 1, WKV_SCORE_TCGEN05 = 2 } wkv_score_impl;
+ * CUDA-core kernels.  Among the tensor-core kernels, shapes with G*alpha <= 128 run in the
+ * pipelined kernel that also gathers (one launch per group); TCGEN05_UNFUSED asks for the
+ * two-launch form instead (score + selection, then the stand-alone gather kernel). */
+typedef enum { WKV_SCORE_AUTO = 0, WKV_SCORE_SIMT = 1, WKV_SCORE_TCGEN05 = 2, WKV_SCORE_TCGEN05_UNFUSED = 3 } wkv_score_impl;
 
 #define WKV_MAX_GROUP_LAYERS 32
 
@@ -327,6 +329,19 @@ int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers,
                             void *const *k_out_layers_dev, void *const *v_out_layers_dev,
                             int32_t *window_idx_dev, int32_t *kept_len_dev, int32_t keep_capacity,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): launches a kernel that does nothing but evaluate
+ * ex2.approx.ftz.f32 (the exponential of Eq. 1 in base 2, the instruction that bounds the score
+ * stage) in eight independent chains per thread, `iters` times.  Timing the launch with CUDA events
+ * and dividing *ex2_per_launch by it gives the device's rate for that instruction, which the
+ * benchmark uses as the special-function floor of the score kernels.
+ *   scratch_dev     DEVICE float[1] (never written in practice)
+ *   blocks, threads grid and block size (threads a multiple of 32, at most 1024)
+ *   ex2_per_launch  HOST out or NULL: exponentials one launch evaluates
+ */
+int wkv_probe_ex2_rate(float *scratch_dev, int32_t blocks, int32_t threads, int32_t iters,
+                       int64_t *ex2_per_launch, void *cuda_stream);
 
 const char *wkv_status_string(int status);
 const char *wkv_last_error_detail(void);

@@ -18,14 +18,14 @@ LIB_PATH = os.path.join(_PKG, "libwkv.so")
 
 WKV_F32, WKV_BF16 = 0, 1
 WKV_TASK_LOCALIZATION, WKV_TASK_AGGREGATION = 0, 1
-WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05 = 0, 1, 2
+WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05, WKV_SCORE_TCGEN05_UNFUSED = 0, 1, 2, 3
 WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_keep_len", "wkv_workspace_sync_words", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
-    "wkv_select_leader_windows", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_select_leader_windows", "wkv_probe_ex2_rate", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
 
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
     L.wkv_compress_group_host.restype = ctypes.c_int
     L.wkv_compress_group_host.argtypes = [sp, i32, vp, sz, vp, vp, sz, vp, vp, sz, vp, vp,
                                           vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.wkv_probe_ex2_rate.restype = ctypes.c_int
+    L.wkv_probe_ex2_rate.argtypes = [vp, i32, i32, i32, ctypes.POINTER(ctypes.c_int64), vp]
     L.wkv_status_string.restype = ctypes.c_char_p
     L.wkv_status_string.argtypes = [ctypes.c_int]
     L.wkv_last_error_detail.restype = ctypes.c_char_p
@@ -409,6 +411,14 @@ def prepare_score_windows(prob: Problem, q_obs, k_leader, window_scores, token_s
                         (prob, q_obs, k_leader, window_scores, token_scores, workspace))
 
 
+def prepare_select_leader_windows(prob: Problem, q_obs_leader, k_leader, window_scores, window_idx, kept_len,
+                                  workspace, lse_obs=None, stream=None) -> PreparedCall:
+    args = (ctypes.byref(prob.shape), _ptr(q_obs_leader), _ptr(k_leader), _ptr(lse_obs), _ptr(window_scores),
+            _ptr(window_idx), _ptr(kept_len), _ptr(workspace), workspace.numel(), _stream(stream))
+    return PreparedCall(lib().wkv_select_leader_windows, "wkv_select_leader_windows", args,
+                        (prob, q_obs_leader, k_leader, lse_obs, window_scores, window_idx, kept_len, workspace))
+
+
 def prepare_select_topk_windows(prob: Problem, window_scores, window_idx, kept_len, stream=None) -> PreparedCall:
     args = (ctypes.byref(prob.shape), _ptr(window_scores), _ptr(window_idx), _ptr(kept_len), _stream(stream))
     return PreparedCall(lib().wkv_select_topk_windows, "wkv_select_topk_windows", args,
@@ -453,6 +463,14 @@ def workspace_sync_words(prob: "Problem", unit: int):
     _check(lib().wkv_workspace_sync_words(ctypes.byref(prob.shape), unit, ctypes.byref(t), ctypes.byref(a)),
            "wkv_workspace_sync_words")
     return int(t.value), int(a.value)
+
+
+def wkv_probe_ex2_rate(scratch, blocks: int, threads: int, iters: int, stream=None) -> int:
+    """Launches the ex2 rate probe; returns the number of exponentials the launch evaluates."""
+    n = ctypes.c_int64(0)
+    _check(lib().wkv_probe_ex2_rate(_ptr(scratch), blocks, threads, iters, ctypes.byref(n), _stream(stream)),
+           "wkv_probe_ex2_rate")
+    return int(n.value)
 
 
 def device_status(workspace) -> int:

@@ -27,6 +27,7 @@
 // Every wait is bounded (mbarriers and the wait for a unit's statistics): on expiry the block sets bit 0 of the
 // status word, drains its own TMA loads, frees its tensor memory and returns.
 #include "tc_common.cuh"
+#include "score_math.cuh"
 #include "topk_block.cuh"
 #include "wkv_internal.cuh"
 
@@ -116,40 +117,6 @@ __device__ __forceinline__ void warp_release(uint64_t *bar, int lane)
 // that count (every waiter of the unit is past its wait by then), clears both words for the next
 // launch and selects.  Bounded: a warp that waits longer than two seconds gives up and sets the
 // block's abort flag.
-__device__ __forceinline__ int ld_acquire_gpu(const int *p)
-{
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void red_release_gpu_add(int *p, int v)
-{
-    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-// one thread: polls until the word has reached `target`; false once the block has given up
-__device__ __forceinline__ bool poll_until_at_least(const int *word, int target, volatile int *abort_flag)
-{
-    unsigned long long t0 = 0;
-    for (uint32_t spin = 1; ld_acquire_gpu(word) < target; ++spin) {
-        if (*abort_flag) return false;
-        if ((spin & 255u) == 0u) {
-            const unsigned long long now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 2 * kWaitLimitNs) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-    return true;
-}
-__device__ __forceinline__ bool warp_wait_arrivals(const int *word, int target, volatile int *abort_flag, int lane)
-{
-    int ok = 1;
-    if (lane == 0) ok = poll_until_at_least(word, target, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
 // geometry of one work item
 struct Item {
     int unit, chunk, b, h;
@@ -166,86 +133,6 @@ __device__ __forceinline__ int tile_at(const Item &im, int u)
 {
     if (!im.reuse) return u;
     return u < kStages ? im.n_tiles - kStages + u : im.n_tiles - 1 - u;
-}
-
-// ---------------------------------------------------------------------------------------------
-// per-element work of the two sweeps
-// ---------------------------------------------------------------------------------------------
-// sweep 1: online-softmax update of one row with 32 more logits (raw dot products; c = log2(e)/sqrt(d))
-__device__ __forceinline__ void stats_update(float (&v)[32], bool fast, int jb, int limit, float c, float &m,
-                                             float &l)
-{
-    if (!fast) {
-#pragma unroll
-        for (int x = 0; x < 32; ++x)
-            if (jb + x > limit) v[x] = -INFINITY;
-    }
-    float g0 = fmaxf(v[0], v[1]), g1 = fmaxf(v[2], v[3]);
-#pragma unroll
-    for (int x = 4; x < 32; x += 4) {
-        g0 = fmaxf(g0, fmaxf(v[x], v[x + 1]));
-        g1 = fmaxf(g1, fmaxf(v[x + 2], v[x + 3]));
-    }
-    const float m_new = fmaxf(m, fmaxf(g0, g1));
-    if (m_new > -INFINITY) {
-        const float mc = m_new * c;
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-        for (int x = 0; x < 32; x += 4) {
-            a0 += fast_exp2(fmaf(v[x], c, -mc));
-            a1 += fast_exp2(fmaf(v[x + 1], c, -mc));
-            a2 += fast_exp2(fmaf(v[x + 2], c, -mc));
-            a3 += fast_exp2(fmaf(v[x + 3], c, -mc));
-        }
-        const float add = (a0 + a1) + (a2 + a3);
-        l = m_new == m ? l + add : l * fast_exp2((m - m_new) * c) + add;
-        m = m_new;
-    }
-}
-// sweep 2: adds exp2(x*c - lse2) of 32 (or 16) rows to the four partial sums of a key
-template <int N>
-__device__ __forceinline__ void score_accumulate(const float (&v)[N], const float *nl_base, float c, float &a0,
-                                                 float &a1, float &a2, float &a3)
-{
-#pragma unroll
-    for (int x = 0; x < N; x += 4) {
-        const float4 nl = *reinterpret_cast<const float4 *>(nl_base + x);
-        a0 += fast_exp2(fmaf(v[x], c, nl.x));
-        a1 += fast_exp2(fmaf(v[x + 1], c, nl.y));
-        a2 += fast_exp2(fmaf(v[x + 2], c, nl.z));
-        a3 += fast_exp2(fmaf(v[x + 3], c, nl.w));
-    }
-}
-
-// Eq. 4 for one window of compile-time length (a power of two) by one thread: a bitonic sorting
-// network in registers (every compare-exchange of a stage is independent of the others, so the
-// thread is not latency-bound), then the p largest are summed in descending order.  Positions
-// beyond `size` (ragged last window) hold -inf and sort to the end.
-template <int omega>
-__device__ __forceinline__ float pool_window_sorted(const float *w, int size, int p)
-{
-    float v[omega];
-#pragma unroll
-    for (int x = 0; x < omega; ++x) v[x] = x < size ? w[x] : -INFINITY;
-#pragma unroll
-    for (int k = 2; k <= omega; k <<= 1)
-#pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1)
-#pragma unroll
-            for (int i = 0; i < omega; ++i) {
-                const int l = i ^ j;
-                if (l > i) {
-                    const float hi = fmaxf(v[i], v[l]), lo = fminf(v[i], v[l]);
-                    const bool descending = (i & k) == 0;
-                    v[i] = descending ? hi : lo;
-                    v[l] = descending ? lo : hi;
-                }
-            }
-    const int p_eff = p < size ? p : size;
-    float acc = 0.f;
-#pragma unroll
-    for (int x = 0; x < omega; ++x) acc += x < p_eff ? v[x] : 0.f;
-    return acc / (float)p_eff;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -577,7 +464,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             }
             __syncthreads();   // `part` is rewritten by the next item
             // release: cumulative over what the block wrote before the barrier above
-            if (threadIdx.x == 0) red_release_gpu_add(a.sync + kSyncTickets + 2 * im.unit + 1, 1);
+            if (threadIdx.x == 0) red_release_gpu_add(a.sync + kSyncTickets + kSyncWordsPerUnit * im.unit + 1, 1);
         }
         if (abort_s) break;
 
@@ -640,7 +527,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                 } else {
                 const int used1 = (im.n + len1 - 1) / len1;   // chunks of the unit that hold keys in sweep 1
                 const bool arrived =
-                    warp_wait_arrivals(a.sync + kSyncTickets + 2 * im.unit + 1, used1, &abort_s, lane);
+                    warp_wait_arrivals(a.sync + kSyncTickets + kSyncWordsPerUnit * im.unit + 1, used1, &abort_s, lane);
                 if (tl < kMergers * q_rows && arrived) {
                     const int r = tl % q_rows, mp = tl / q_rows;
                     float M = -INFINITY, sum = 0.f;
@@ -739,7 +626,7 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
             // chunk is usually a short one, so its block is done early and the selection does not sit
             // on the path of a block that the next wave is waiting for.  The other blocks only count
             // themselves, without waiting for an answer.
-            int *ticket = a.sync + kSyncTickets + 2 * im.unit;
+            int *ticket = a.sync + kSyncTickets + kSyncWordsPerUnit * im.unit;
             if (im.chunk != used2 - 1) {
                 if (a.window_idx) {
                     __syncthreads();

@@ -31,6 +31,21 @@ struct TopkSmem {
     int cand_total, n_cand;     // keys in the chosen bin; candidates collected for the direct finish
 };
 
+// The NT threads that take part are threads TID0 .. TID0 + NT - 1 of the block.  BAR = 0: they are the
+// whole block and synchronise with the block barrier; BAR > 0: they are a subset of the block's warps
+// and synchronise on named barrier BAR (the rest of the block runs on independently).
+template <int TID0>
+__device__ __forceinline__ int topk_tid()
+{
+    return (int)threadIdx.x - TID0;
+}
+template <int NT, int BAR>
+__device__ __forceinline__ void topk_sync()
+{
+    if (BAR == 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
 // larger float <=> larger key; -0 and +0 map to the same key
 __device__ __forceinline__ unsigned topk_order_key(float f)
 {
@@ -53,14 +68,14 @@ __device__ __forceinline__ int topk_warp_scan(int v, int lane)   // inclusive
 // written per warp, one barrier, then every warp adds up the totals of the warps before it with a
 // warp-reduce instruction.  `warp_sums` (32 words) must not be in use by a scan that some thread
 // of the block may not have left yet: alternate between two slots.
-template <int NT>
+template <int NT, int BAR, int TID0>
 __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total)
 {
     constexpr int kWarps = NT / 32;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = topk_tid<TID0>() & 31, warp = topk_tid<TID0>() >> 5;
     const int incl = topk_warp_scan(v, lane);
     if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
+    topk_sync<NT, BAR>();
     const int wt = lane < kWarps ? warp_sums[lane] : 0;
     total = __reduce_add_sync(0xffffffffu, wt);
     return __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0) + incl - v;
@@ -72,15 +87,15 @@ __device__ __forceinline__ int topk_block_scan(int v, int *warp_sums, int &total
 // Thread t owns the windows [t*E, (t+1)*E), E = ceil(kw / NT).  With E <= REGS (4 or 8) the keys
 // are read once and stay in registers through the radix passes and the compaction (one trip to L2
 // instead of several); REGS = 0: longer lists are re-read.
-template <int NT, int REGS>
+template <int NT, int REGS, int BAR, int TID0>
 __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, int kw, int k, int *out,
                                                  int *kept_len_out, int n, int alpha, int omega, int obs_rows)
 {
     constexpr int kWarps = NT / 32;
     static_assert(NT % 32 == 0 && NT >= kTopkDirect, "block size");
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = topk_tid<TID0>() & 31, warp = topk_tid<TID0>() >> 5;
     const int E = (kw + NT - 1) / NT;
-    const int w_lo = min(kw, (int)threadIdx.x * E), w_hi = min(kw, w_lo + E);
+    const int w_lo = min(kw, (int)topk_tid<TID0>() * E), w_hi = min(kw, w_lo + E);
     constexpr bool IN_REGS = REGS > 0;
     constexpr int kTopkRegs = IN_REGS ? REGS : 1;
     unsigned keys[kTopkRegs];
@@ -105,14 +120,14 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     // from it are resolved, 9 at a time from the top (window scores share sign and most of the
     // exponent: typically one pass), until at most kTopkDirect candidates share the prefix; those
     // are ranked against each other directly.
-    if (threadIdx.x == 0) {
+    if (topk_tid<TID0>() == 0) {
         sm.prefix = 0u;
         sm.remaining = k;
         sm.last_selected = 0;
         sm.cand_total = kw;
         sm.n_cand = 0;
     }
-    for (int x = threadIdx.x; x < kTopkBins; x += NT) sm.hist[x] = 0;
+    for (int x = topk_tid<TID0>(); x < kTopkBins; x += NT) sm.hist[x] = 0;
     unsigned kmin, kmax;
     {
         unsigned lo = 0xffffffffu, hi = 0u;
@@ -126,7 +141,7 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
             sm.warp_min[warp] = lo;
             sm.warp_max[warp] = hi;
         }
-        __syncthreads();
+        topk_sync<NT, BAR>();
         kmin = __reduce_min_sync(0xffffffffu, lane < kWarps ? sm.warp_min[lane] : 0xffffffffu);
         kmax = __reduce_max_sync(0xffffffffu, lane < kWarps ? sm.warp_max[lane] : 0u);
     }
@@ -150,10 +165,10 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
                 const unsigned rk = key - kmin;
                 if ((rk & mask) == prefix) sm.cand[slot++] = rk;
             });
-            __syncthreads();
+            topk_sync<NT, BAR>();
             const int n_cand = sm.n_cand;
-            if ((int)threadIdx.x < n_cand) {
-                const unsigned my = sm.cand[threadIdx.x];
+            if ((int)topk_tid<TID0>() < n_cand) {
+                const unsigned my = sm.cand[topk_tid<TID0>()];
                 int gt = 0, eq = 0;
                 for (int j = 0; j < n_cand; ++j) {
                     const unsigned o = sm.cand[j];
@@ -165,7 +180,7 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
                     sm.remaining = remaining - gt;
                 }
             }
-            __syncthreads();
+            topk_sync<NT, BAR>();
             break;
         }
         const int low = top > kTopkDigit ? top - kTopkDigit : 0;
@@ -174,7 +189,7 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
             const unsigned rk = key - kmin;
             if ((rk & mask) == prefix) atomicAdd(&sm.hist[(rk >> low) & digit_mask], 1);
         });
-        __syncthreads();
+        topk_sync<NT, BAR>();
         if (warp == 0) {
             // the bin (from the top) in which the count reaches `remaining`: lane l holds bins 16 l .. 16 l + 15
             int c[16], mine = 0;
@@ -213,7 +228,7 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
         }
         mask |= digit_mask << low;
         top = low;
-        __syncthreads();
+        topk_sync<NT, BAR>();
     }
     const unsigned thr = sm.prefix + kmin;
     const int need_eq = sm.remaining;
@@ -238,15 +253,15 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     if (IN_REGS) {
         // at most NT * 8 < 2^15 windows: both counts travel through one scan
         int total;
-        const int both = topk_block_scan<NT>((n_eq << 16) | n_gt, sm.warp_sums[0], total);
+        const int both = topk_block_scan<NT, BAR, TID0>((n_eq << 16) | n_gt, sm.warp_sums[0], total);
         eq_rank = both >> 16;
         pos = (both & 0xffff) + (eq_rank < need_eq ? eq_rank : need_eq);
     } else {
         int eq_total, sel_total;
-        eq_rank = topk_block_scan<NT>(n_eq, sm.warp_sums[0], eq_total);
+        eq_rank = topk_block_scan<NT, BAR, TID0>(n_eq, sm.warp_sums[0], eq_total);
         int n_eq_taken = need_eq - eq_rank;
         n_eq_taken = n_eq_taken < 0 ? 0 : (n_eq_taken > n_eq ? n_eq : n_eq_taken);
-        pos = topk_block_scan<NT>(n_gt + n_eq_taken, sm.warp_sums[1], sel_total);
+        pos = topk_block_scan<NT, BAR, TID0>(n_gt + n_eq_taken, sm.warp_sums[1], sel_total);
     }
     auto emit = [&](int e, unsigned key) {
         bool sel = key > thr;
@@ -266,32 +281,32 @@ __device__ __forceinline__ void select_topk_impl(TopkSmem &sm, const float *sc, 
     } else {
         for (int e = 0; w_lo + e < w_hi; ++e) emit(e, key_at(e));
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
+    topk_sync<NT, BAR>();
+    if (topk_tid<TID0>() == 0) {
         const int n_r = n - alpha;
         const int last_size = n_r - (kw - 1) * omega;     // real size of the last window
         *kept_len_out = k * omega - (sm.last_selected ? omega - last_size : 0) + obs_rows;
     }
 }
 
-template <int NT>
+template <int NT, int BAR = 0, int TID0 = 0>
 __device__ void select_topk_block(TopkSmem &sm, const float *sc, int kw, int k, int k_max, int *out,
                                   int *kept_len_out, int n, int alpha, int omega)
 {
     static_assert(NT % 32 == 0 && NT <= 1024, "block size");
-    for (int x = (k > 0 ? k : 0) + threadIdx.x; x < k_max; x += NT) out[x] = -1;
+    for (int x = (k > 0 ? k : 0) + topk_tid<TID0>(); x < k_max; x += NT) out[x] = -1;
     const int obs_rows = n < alpha ? n : alpha;
     if (k <= 0) {
-        if (threadIdx.x == 0) *kept_len_out = obs_rows;
+        if (topk_tid<TID0>() == 0) *kept_len_out = obs_rows;
         return;
     }
     const int per_thread = (kw + NT - 1) / NT;
     if (per_thread <= 4)
-        select_topk_impl<NT, 4>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+        select_topk_impl<NT, 4, BAR, TID0>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
     else if (per_thread <= 8)
-        select_topk_impl<NT, 8>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+        select_topk_impl<NT, 8, BAR, TID0>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
     else
-        select_topk_impl<NT, 0>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
+        select_topk_impl<NT, 0, BAR, TID0>(sm, sc, kw, k, out, kept_len_out, n, alpha, omega, obs_rows);
 }
 
 }  // namespace wkv

@@ -35,11 +35,13 @@ Workspace plan_workspace(const KShape &ks)
     w.n_stat_chunks = (ks.max_seqlen + kStatChunk - 1) / kStatChunk;
     const int tc_chunks = tc_plan((int)units, ks.max_seqlen, ks.d).chunks_per_unit;
     if (tc_chunks > w.n_stat_chunks) w.n_stat_chunks = tc_chunks;
+    const int pipe_chunks = pipe_plan((int)units, ks.max_seqlen, ks.d).chunks_per_unit;
+    if (pipe_chunks > w.n_stat_chunks) w.n_stat_chunks = pipe_chunks;
     size_t off = 0;
     w.status_off = off;
     off = 64;
     w.sync_off = off;
-    off = align_up(off + (16 + 2 * (size_t)units) * sizeof(int), 256);
+    off = align_up(off + (kSyncTickets + kSyncWordsPerUnit * (size_t)units) * sizeof(int), 256);
     w.stats_off = off;
     off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
     w.lse_off = off;
@@ -84,7 +86,7 @@ int resolve(const wkv_shape *s, KShape &ks)
         set_error_detail("task %d unknown", s->task);
         return WKV_ERR_SHAPE;
     }
-    if (s->score_impl < WKV_SCORE_AUTO || s->score_impl > WKV_SCORE_TCGEN05 || s->reserved != 0) {
+    if (s->score_impl < WKV_SCORE_AUTO || s->score_impl > WKV_SCORE_TCGEN05_UNFUSED || s->reserved != 0) {
         set_error_detail("score_impl %d / reserved %d invalid", s->score_impl, s->reserved);
         return WKV_ERR_SHAPE;
     }
@@ -197,8 +199,9 @@ static int check_workspace(const Workspace &ws, const void *workspace, size_t by
 static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace &ws, bool &use_tc)
 {
     const bool tc_ok = score_tc_supported(ks, s->dtype);
-    if (s->score_impl == WKV_SCORE_TCGEN05 && !tc_ok) {
-        set_error_detail("tensor-core score kernels need bf16, head_dim 64/128 and G*alpha <= 256");
+    if ((s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_UNFUSED) && !tc_ok) {
+        set_error_detail("tensor-core score kernels need bf16, head_dim 64/128 and G*alpha <= 256 on a device of "
+                         "compute capability 10");
         return WKV_ERR_UNSUPPORTED;
     }
     use_tc = tc_ok && s->score_impl != WKV_SCORE_SIMT;
@@ -215,8 +218,9 @@ static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace
 
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
              float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
-             cudaStream_t stream, const float *lse_obs)
+             cudaStream_t stream, const float *lse_obs, const PipeGather *gather, bool *gathered)
 {
+    if (gathered) *gathered = false;
     if (!aligned16(q) || !aligned16(k)) {
         set_error_detail("q_obs / k_leader not 16-byte aligned");
         return WKV_ERR_ALIGN;
@@ -225,10 +229,20 @@ int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const vo
     int st = pick_score_impl(s, ks, ws, use_tc);
     if (st != WKV_OK) return st;
     if (use_tc) {
-        st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream,
-                             lse_obs);
+        const bool forced = s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_UNFUSED;
+        st = WKV_ERR_UNSUPPORTED;
+        if (s->score_impl != WKV_SCORE_TCGEN05_UNFUSED && group_pipeline_supported(ks, s->dtype)) {
+            // one launch for scoring, selection and (when asked and possible) the gather
+            const bool fuse = gather && window_idx && group_pipeline_can_gather(ks, elem_bytes(s->dtype), gather->n_tensors);
+            st = launch_group_pipeline(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws,
+                                       stream, lse_obs, fuse ? gather : nullptr);
+            if (st == WKV_OK && fuse && gathered) *gathered = true;
+        }
+        if (st == WKV_ERR_UNSUPPORTED)
+            st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream,
+                                 lse_obs);
         // a key layout that no tensor map can describe is served by the CUDA-core kernels
-        if (st != WKV_ERR_UNSUPPORTED || s->score_impl == WKV_SCORE_TCGEN05) return st;
+        if (st != WKV_ERR_UNSUPPORTED || forced) return st;
         if (score_simt_smem_bytes(ks, ws.r_pad) > 227u * 1024u) return st;
     }
     st = check_cuda(launch_score_simt(ks, s->dtype, q, k, window_scores, token_scores, workspace, ws, stream,
@@ -327,7 +341,7 @@ int wkv_workspace_sync_words(const wkv_shape *s, int32_t unit, size_t *ticket_by
         return WKV_ERR_SHAPE;
     }
     const Workspace ws = plan_workspace(ks);
-    const size_t ticket = ws.sync_off + sizeof(int) * ((size_t)kSyncTickets + 2 * (size_t)unit);
+    const size_t ticket = ws.sync_off + sizeof(int) * ((size_t)kSyncTickets + kSyncWordsPerUnit * (size_t)unit);
     if (ticket_byte_offset) *ticket_byte_offset = ticket;
     if (arrival_byte_offset) *arrival_byte_offset = ticket + sizeof(int);
     return WKV_OK;
@@ -519,9 +533,15 @@ int wkv::compress_group_entry(const wkv_shape *s, int32_t n_layers, const void *
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float *scores = window_scores ? window_scores
                                   : reinterpret_cast<float *>(static_cast<char *>(workspace) + ws.scores_off);
+    PipeGather pg;
+    pg.n_tensors = n_tensors;
+    pg.tab = &tab;
+    pg.cu_out = cu_seqlens_out;
+    pg.keep_capacity = keep_capacity;
+    bool gathered = false;
     st = do_score(s, ks, ws, q_obs_leader, k_layers[0], scores, nullptr, window_idx, kept_len, workspace, stream,
-                  lse_obs);
-    if (st != WKV_OK) return st;
+                  lse_obs, &pg, &gathered);
+    if (st != WKV_OK || gathered) return st;
     return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
                                     keep_capacity, stream),
                       "gather kernel");

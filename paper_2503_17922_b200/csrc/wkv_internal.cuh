@@ -75,7 +75,7 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
     size_t status_off;   // int: device status word, only ever OR-ed by the kernels (0 = no error)
-    size_t sync_off;     // int [16 + 2 * units]: per unit a ticket and a count of sweep-1 arrivals (self-resetting)
+    size_t sync_off;     // int [kSyncTickets + kSyncWordsPerUnit * units], self-resetting
     size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
     size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
     size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none
@@ -84,9 +84,11 @@ struct Workspace {
     int r_pad;
 };
 
-// words of the synchronisation area before the per-unit words: unit u owns sync[kSyncTickets + 2u]
-// (ticket) and sync[kSyncTickets + 2u + 1] (arrivals of the statistics sweep)
+// words of the synchronisation area before the per-unit words; unit u owns four words from
+// sync[kSyncTickets + 4u]: ticket count, arrivals of the statistics sweep, "selection published" flag
+// and gather job counter (the last two only in the kernel that also gathers)
 constexpr int kSyncTickets = 16;
+constexpr int kSyncWordsPerUnit = 4;
 
 // per-device host state (kernel attributes, device properties) is kept for this many device ordinals
 constexpr int kMaxDevices = 64;
@@ -129,6 +131,31 @@ __host__ __device__ inline TcPlan tc_plan(int units, int max_seqlen, int head_di
     p.chunks_per_unit = a > b ? a : b;
     return p;
 }
+// The pipelined group kernel takes the units in waves too, but keeps TWO waves in flight (the
+// statistics sweep runs one wave ahead of the scoring sweep), so two waves' keys share the L2 budget;
+// with at least two units it always makes at least two waves, so that the gather of one wave's rows
+// can run beside the scoring of the next.
+struct PipePlan {
+    int units_per_wave, chunks_per_unit, skew;
+};
+__host__ __device__ inline PipePlan pipe_plan(int units, int max_seqlen, int head_dim)
+{
+    PipePlan p;
+    const long long unit_bytes = (long long)max_seqlen * head_dim * 2;
+    const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
+    const int min_chunks = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
+    long long upw = (kTcWaveBytes / 2) / (unit_bytes > 0 ? unit_bytes : 1);
+    if (upw > kTcTargetBlocks / min_chunks) upw = kTcTargetBlocks / min_chunks;
+    if (upw > (units + 1) / 2) upw = (units + 1) / 2;
+    if (upw < 1) upw = 1;
+    p.units_per_wave = (int)upw;
+    p.skew = units > p.units_per_wave ? 1 : 0;
+    int a = kTcTargetBlocks / p.units_per_wave;
+    if (a < 1) a = 1;
+    if (a > max_tiles) a = max_tiles;
+    p.chunks_per_unit = a > min_chunks ? a : min_chunks;
+    return p;
+}
 // keys per block when `n_keys` keys are split over `chunks` blocks in whole tiles, rounded up to a
 // multiple of `align` (1 for the statistics sweep, omega for the scoring sweep)
 __host__ __device__ inline int tc_chunk_len(int n_keys, int chunks, int align)
@@ -156,6 +183,20 @@ bool score_tc_supported(const KShape &ks, int dtype);
 int launch_score_tc(const KShape &ks, const void *q, const void *k,
                     float *window_scores, float *token_scores, int *window_idx, int *kept_len,
                     void *workspace, const Workspace &ws, cudaStream_t stream, const float *lse_obs = nullptr);
+// The pipelined group kernel (score_pipe.cu): scoring, selection and, with `gather`, the shared-index
+// gather of every layer in one launch.  R <= 128 only.
+struct LayerTable;
+struct PipeGather {
+    int n_tensors;
+    const LayerTable *tab;
+    const int *cu_out;
+    int keep_capacity;
+};
+bool group_pipeline_supported(const KShape &ks, int dtype);
+bool group_pipeline_can_gather(const KShape &ks, int elem_bytes, int n_tensors);
+int launch_group_pipeline(const KShape &ks, const void *q, const void *k, float *window_scores, float *token_scores,
+                          int *window_idx, int *kept_len, void *workspace, const Workspace &ws, cudaStream_t stream,
+                          const float *lse_obs, const PipeGather *gather);
 cudaError_t launch_topk(const KShape &ks, const float *window_scores, int *window_idx, int *kept_len,
                         cudaStream_t stream);
 
@@ -200,9 +241,12 @@ __device__ inline float pool_top_p(const float *w, int size, int p)
 int resolve(const wkv_shape *s, KShape &ks);            // validates the shape, fills the kernel-side copy
 int check_cuda(cudaError_t e, const char *what);         // cudaError_t -> wkv_status with detail
 // scoring; with window_idx / kept_len non-null also the selection (one launch on the tensor-core path)
+// `gather` non-null: the caller wants the layers gathered as well; *gathered tells whether the launch
+// that scored has done it (else the caller launches the gather kernel)
 int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const void *q, const void *k,
              float *window_scores, float *token_scores, int *window_idx, int *kept_len, void *workspace,
-             cudaStream_t stream, const float *lse_obs = nullptr);
+             cudaStream_t stream, const float *lse_obs = nullptr, const PipeGather *gather = nullptr,
+             bool *gathered = nullptr);
 
 void count_launches(int n);
 uint64_t launches_so_far();

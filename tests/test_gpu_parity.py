@@ -138,7 +138,7 @@ def test_group_plan_replays_the_group_call():
         before = binding.wkv_launch_count()
         plan.launch()
         torch.cuda.synchronize()
-        assert binding.wkv_launch_count() - before >= 2
+        assert binding.wkv_launch_count() - before >= 1          # one launch when the pipelined kernel also gathers
         assert binding.device_status(work) == 0
         ref = pu.run_gpu_group(w, grp)
         np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), ref["window_idx"])
@@ -473,7 +473,7 @@ def _run_host_entry(w, grp):
                                     out["k_out"], out["v_out"], out["window_idx"], out["kept_len"],
                                     out["keep_capacity"], work)
     # the call returns after synchronising its stream: the host buffers are complete here
-    assert binding.wkv_launch_count() - before >= 2
+    assert binding.wkv_launch_count() - before >= 1
     assert binding.device_status(work) == 0
     return {"prob": prob, "window_idx": h_idx.numpy().copy(), "kept_len": h_kept.numpy().copy(),
             "k_out": [binding.to_host_bits(t) for t in h_k_out], "v_out": [binding.to_host_bits(t) for t in h_v_out],
@@ -505,7 +505,7 @@ def test_launches_are_counted_and_errors_raise():
     w = small()
     before = binding.wkv_launch_count()
     pu.run_gpu_group(w, wl.make_group(w, 0))
-    assert binding.wkv_launch_count() - before >= 2     # fused score+selection launch, gather launch
+    assert binding.wkv_launch_count() - before >= 1     # one pipelined launch, or score+selection and gather
     prob = binding.Problem.from_workload(w)
     with pytest.raises(binding.WkvError):
         binding.wkv_score_windows(prob, None, None, None, None, prob.alloc_workspace())
