@@ -248,7 +248,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=40)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
-    ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05", "unfused"])
+    ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05", "pipelined"])
     ap.add_argument("--groups", type=int, default=0, help="distinct groups kept on the device (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -280,10 +280,10 @@ def main() -> None:
 
     w = pick_workload(args.workload)
     impl = {"auto": binding.WKV_SCORE_AUTO, "simt": binding.WKV_SCORE_SIMT,
-            "tcgen05": binding.WKV_SCORE_TCGEN05, "unfused": binding.WKV_SCORE_TCGEN05_UNFUSED}[args.score_impl]
+            "tcgen05": binding.WKV_SCORE_TCGEN05, "pipelined": binding.WKV_SCORE_TCGEN05_PIPELINED}[args.score_impl]
     prob = binding.Problem.from_workload(w, score_impl=impl)
-    prob_unfused = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05_UNFUSED) \
-        if (impl == binding.WKV_SCORE_AUTO and w.dtype == "bf16") else None
+    prob_pipe = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05_PIPELINED) \
+        if (impl == binding.WKV_SCORE_AUTO and w.dtype == "bf16" and w.rows <= 128) else None
     alg = algorithmic_bytes(w, prob)
     tokens = alg["tokens"]
     warmup = max(args.warmup, 3)
@@ -317,9 +317,9 @@ def main() -> None:
     leader_calls = [binding.prepare_select_leader_windows(prob, d["q"], d["k"][0], out["window_scores"],
                                                           out["window_idx"], out["kept_len"], work, stream=stream)
                     for d in dev_groups]
-    unfused_calls = None
-    if prob_unfused is not None:
-        unfused_calls = [binding.prepare_compress_group(prob_unfused, d["q"], d["k"], d["v"], out["k_out"],
+    pipe_calls = None
+    if prob_pipe is not None:
+        pipe_calls = [binding.prepare_compress_group(prob_pipe, d["q"], d["k"], d["v"], out["k_out"],
                                                         out["v_out"], out["window_scores"], out["window_idx"],
                                                         out["kept_len"], work, keep_capacity=cap, stream=stream)
                          for d in dev_groups]
@@ -422,7 +422,7 @@ def main() -> None:
         ms_fused = time_stage(group_calls)                 # the group call's launch(es), graph replay
         ms_score = time_stage(score_calls)                 # scores and pooling only
         ms_score_select = time_stage(leader_calls)         # scores, pooling and selection in one launch, timed directly
-        ms_unfused = time_stage(unfused_calls) if unfused_calls else None   # two-launch form of the group
+        ms_pipe = time_stage(pipe_calls) if pipe_calls else None   # the opt-in single-launch form of the group
         # the special-function rate of this GPU, measured: 148 x 4 blocks of 1024 threads, 8 chains each
         probe_scratch = torch.zeros(4, dtype=torch.float32, device="cuda")
         binding.wkv_probe_ex2_rate(probe_scratch, 592, 1024, 64, stream=stream)
@@ -535,7 +535,7 @@ def main() -> None:
             "gpu_launches": int(launches),
             "path_hbm_frac": path_frac,
             "path_algorithmic_bytes": alg["total"],
-            "stages_ms": {"group_graph_replay": ms_fused, "group_two_launch_form": ms_unfused,
+            "stages_ms": {"group_graph_replay": ms_fused, "group_pipelined_single_launch_form": ms_pipe,
                           "score_select_one_launch": ms_score_select,
                           "score_only": ms_score, "select_standalone": ms_select, "gather_standalone": ms_gather,
                           "group_given_lse_graph_replay": ms_given_lse,

@@ -74,10 +74,13 @@ typedef enum { WKV_F32 = 0, WKV_BF16 = 1 } wkv_dtype;
 typedef enum { WKV_TASK_LOCALIZATION = 0, WKV_TASK_AGGREGATION = 1 } wkv_task;
 /* which score kernel family to use: AUTO picks the tensor-core (tcgen05) kernels
  * for bf16 inputs with head_dim 64 or 128 and G*alpha <= 256, else the plain
- * CUDA-core kernels.  Among the tensor-core kernels, shapes with G*alpha <= 128 run in the
- * pipelined kernel that also gathers (one launch per group); TCGEN05_UNFUSED asks for the
- * two-launch form instead (score + selection, then the stand-alone gather kernel). */
-typedef enum { WKV_SCORE_AUTO = 0, WKV_SCORE_SIMT = 1, WKV_SCORE_TCGEN05 = 2, WKV_SCORE_TCGEN05_UNFUSED = 3 } wkv_score_impl;
+ * CUDA-core kernels.  TCGEN05 forces the tensor-core kernels (score + selection in one launch,
+ * the gather in a second one).  TCGEN05_PIPELINED asks for the single-launch form instead
+ * (G*alpha <= 128 only): statistics sweep one wave ahead of the scoring sweep and the gather done
+ * by bulk copies inside the same kernel.  It gives the same results and is slower on every
+ * configuration measured so far, so AUTO never picks it; it is kept as an option for
+ * measurements. */
+typedef enum { WKV_SCORE_AUTO = 0, WKV_SCORE_SIMT = 1, WKV_SCORE_TCGEN05 = 2, WKV_SCORE_TCGEN05_PIPELINED = 3 } wkv_score_impl;
 
 #define WKV_MAX_GROUP_LAYERS 32
 
@@ -342,6 +345,16 @@ int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers,
  */
 int wkv_probe_ex2_rate(float *scratch_dev, int32_t blocks, int32_t threads, int32_t iters,
                        int64_t *ex2_per_launch, void *cuda_stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): the rate of the cross-lane column sum a single-sweep
+ * score kernel would need (a warp holds a 32 x 32 block of values, one row per lane, and sums its
+ * columns over the lanes with 31 shuffle-and-add steps), in block elements per launch.  Compared with
+ * wkv_probe_ex2_rate it tells whether replacing the second sweep's exponentials by such a reduction
+ * could be faster.  Arguments as wkv_probe_ex2_rate.
+ */
+int wkv_probe_colsum_rate(float *scratch_dev, int32_t blocks, int32_t threads, int32_t iters,
+                          int64_t *elements_per_launch, void *cuda_stream);
 
 const char *wkv_status_string(int status);
 const char *wkv_last_error_detail(void);

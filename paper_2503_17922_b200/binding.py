@@ -18,14 +18,14 @@ LIB_PATH = os.path.join(_PKG, "libwkv.so")
 
 WKV_F32, WKV_BF16 = 0, 1
 WKV_TASK_LOCALIZATION, WKV_TASK_AGGREGATION = 0, 1
-WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05, WKV_SCORE_TCGEN05_UNFUSED = 0, 1, 2, 3
+WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05, WKV_SCORE_TCGEN05_PIPELINED = 0, 1, 2, 3
 WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
     "wkv_num_windows", "wkv_num_selected", "wkv_keep_len", "wkv_workspace_sync_words", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
     "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
-    "wkv_select_leader_windows", "wkv_probe_ex2_rate", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
+    "wkv_select_leader_windows", "wkv_probe_ex2_rate", "wkv_probe_colsum_rate", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
 ]
 
@@ -123,6 +123,8 @@ def lib() -> ctypes.CDLL:
                                           vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     L.wkv_probe_ex2_rate.restype = ctypes.c_int
     L.wkv_probe_ex2_rate.argtypes = [vp, i32, i32, i32, ctypes.POINTER(ctypes.c_int64), vp]
+    L.wkv_probe_colsum_rate.restype = ctypes.c_int
+    L.wkv_probe_colsum_rate.argtypes = [vp, i32, i32, i32, ctypes.POINTER(ctypes.c_int64), vp]
     L.wkv_status_string.restype = ctypes.c_char_p
     L.wkv_status_string.argtypes = [ctypes.c_int]
     L.wkv_last_error_detail.restype = ctypes.c_char_p
@@ -470,6 +472,14 @@ def wkv_probe_ex2_rate(scratch, blocks: int, threads: int, iters: int, stream=No
     n = ctypes.c_int64(0)
     _check(lib().wkv_probe_ex2_rate(_ptr(scratch), blocks, threads, iters, ctypes.byref(n), _stream(stream)),
            "wkv_probe_ex2_rate")
+    return int(n.value)
+
+
+def wkv_probe_colsum_rate(scratch, blocks: int, threads: int, iters: int, stream=None) -> int:
+    """Launches the cross-lane column-sum probe; returns the number of block elements it reduces."""
+    n = ctypes.c_int64(0)
+    _check(lib().wkv_probe_colsum_rate(_ptr(scratch), blocks, threads, iters, ctypes.byref(n), _stream(stream)),
+           "wkv_probe_colsum_rate")
     return int(n.value)
 
 

@@ -19,9 +19,12 @@
 //     windows of every layer's K and V with bulk asynchronous copies (global -> shared -> global,
 //     4 KB slots, L2 evict-first so that the keys of the wave still to be scored stay in L2).  Jobs are
 //     handed out through one counter per unit, so when the scoring is over the producer warp joins in
-//     with the idle tile ring as 24 more slots and the tail of the gather runs at the copy rate.
-// Two Q images live in shared memory (wave parity), so that the sweep over wave w and the sweep over
-// wave w-1 alternate without reloading them.
+//     with the idle tile ring as 32 more slots and the tail of the gather runs at the copy rate.
+// The Q image of an item's unit is fetched by TMA when the producer reaches the item (32 KB out of L2,
+// behind the accumulators the compute warps still have to work through).
+// The per-chunk row statistics travel between blocks as self-validating 8-byte entries (the low
+// mantissa bit of the sum marks an entry as written; the area is zero between launches), so that
+// publishing them needs no fence and reading them no counter.
 //
 // Every wait is bounded (mbarriers, arrival counts, selection flags): on expiry the block sets bit 0
 // of the status word, lets its own asynchronous copies land, frees its tensor memory and returns.
@@ -40,7 +43,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kStages = 3;                               // key tiles in flight
+constexpr int kStages = 4;                               // key tiles in flight
 constexpr int kBufs = 4;                                 // accumulator buffers of 128 columns
 constexpr int kTile = kTcTileKeys;
 constexpr int kRegion = kTile * 128;                     // bytes of one 64-column block of a key tile
@@ -58,7 +61,7 @@ constexpr int kBarCompute = 3;                           // named barrier of the
 
 struct PipeArgs {
     KShape s;
-    float2 *stats;          // [units][n_stat_chunks][r_pad]
+    unsigned long long *pstats;   // [units][n_stat_chunks][128] self-validating (max, sum) entries, zero between launches
     float *window_scores;
     float *token_scores;
     const float *lse_obs;
@@ -66,7 +69,7 @@ struct PipeArgs {
     int *kept_len;
     int *status;
     int *sync;
-    int n_stat_chunks, r_pad;
+    int n_stat_chunks;
     int chunks_per_unit, units_per_wave, n_waves, skew;
     int kblocks;            // head_dim / 64
     int slot_tok, slot_h, slot_b;
@@ -92,7 +95,7 @@ __device__ __forceinline__ uint8_t *align_1024(uint8_t *p)
 struct PipeBarriers {
     uint64_t full[kStages], empty[kStages];
     uint64_t tfull[kBufs], tempty[kBufs];
-    uint64_t qfull[2], qfree[2];
+    uint64_t qfull, qfree;
     uint64_t copy[kCopyWarps][kCopySlots];
     uint64_t tail[kTailSlotsMax];
 };
@@ -116,6 +119,35 @@ __device__ __forceinline__ void compute_sync()
 __device__ __forceinline__ void st_release_gpu(int *p, int v)
 {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// ---- self-validating statistics entries ----------------------------------------------------------
+// One 8-byte word per (unit, chunk, row): the row's maximum (times log2(e)/sqrt(d)) in the low half and
+// its sum of exponentials in the high half, with the lowest mantissa bit of the sum forced to one so
+// that a written entry is never all zero (an empty row's sum 0 becomes the smallest denormal).  The
+// reader clears that bit again: the sum loses at most one unit in the last place.  Written and read
+// with single 64-bit accesses, so an entry is seen whole or not at all.
+__device__ __forceinline__ unsigned long long stat_pack(float m, float sum)
+{
+    const unsigned hi = sum == 0.f ? 1u : (__float_as_uint(sum) | 1u);
+    return ((unsigned long long)hi << 32) | (unsigned long long)__float_as_uint(m);
+}
+__device__ __forceinline__ bool stat_unpack(unsigned long long w, float2 &out)
+{
+    const unsigned hi = (unsigned)(w >> 32);
+    out.x = __uint_as_float((unsigned)w);
+    out.y = __uint_as_float(hi & ~1u);
+    return hi != 0u;
+}
+__device__ __forceinline__ void st_relaxed_gpu_u64(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
 }
 
 // ---- bulk asynchronous copies (no multicast) ----------------------------------------------------
@@ -151,7 +183,6 @@ struct Entry {
     int n, n_r;
     long long off;
     int j_begin, j_end, n_tiles;
-    int qbuf;
 };
 struct Cursor {
     int step, phase, j;
@@ -200,7 +231,6 @@ __device__ __forceinline__ bool next_entry(const PipeArgs &a, Cursor &c, Entry &
                 e.j_begin = e.chunk * len;
                 e.j_end = min(n_keys, e.j_begin + len);
                 e.n_tiles = (e.n_r > 0 && e.j_end > e.j_begin) ? (e.j_end - e.j_begin + kTile - 1) / kTile : 0;
-                e.qbuf = wave & 1;
                 return true;
             }
         }
@@ -215,12 +245,12 @@ __device__ __forceinline__ bool next_entry(const PipeArgs &a, Cursor &c, Entry &
     }
 }
 
-// Which unit's queries each of the two Q images holds; producer and MMA warp keep identical copies of
-// this state by walking the same list, so both know when an image is (re)loaded.
+// Which unit's queries the Q image holds; producer and MMA warp keep identical copies of this state
+// by walking the same list, so both know when the image is (re)loaded.
 struct QState {
-    int unit[2];
-    uint32_t loads[2];   // images loaded into the buffer so far
-    uint32_t uses[2];    // items that have multiplied against the buffer so far
+    int unit;
+    uint32_t loads;      // images loaded so far
+    uint32_t frees;      // hand-backs of the image (MMA warp -> producer) so far
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -378,7 +408,7 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     const int q_img_bytes = a.kblocks * kQRegion;
     const int stage_bytes = a.kblocks * kRegion;
     uint8_t *q_img0 = align_1024(smem_raw);
-    uint8_t *k_stage0 = q_img0 + 2 * q_img_bytes;
+    uint8_t *k_stage0 = q_img0 + q_img_bytes;
     uint8_t *copy_ring = k_stage0 + kStages * stage_bytes;
     const int ksteps = s.d / 16;
     const bool gathers = a.n_tensors > 0 && a.window_idx != nullptr;
@@ -392,18 +422,16 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
             mbar_init(&bar.tfull[i], 1);
             mbar_init(&bar.tempty[i], 4);     // one arrival per warp of the group
         }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&bar.qfull[i], 1);
-            mbar_init(&bar.qfree[i], 1);
-        }
+        mbar_init(&bar.qfull, 1);
+        mbar_init(&bar.qfree, 1);
         for (int i = 0; i < kCopyWarps * kCopySlots; ++i) mbar_init(&bar.copy[0][0] + i, 1);
         for (int i = 0; i < kTailSlotsMax; ++i) mbar_init(&bar.tail[i], 1);
         fence_barrier_init();
         abort_s = 0;
     }
     if (warp == 1) tmem_alloc(&tmem_base_s, tmem_cols);
-    // rows of the Q images that no load ever writes (padding up to the image height) must read as zero
-    for (int i = threadIdx.x; i < 2 * q_img_bytes / 16; i += kThreads)
+    // rows of the Q image that no load ever writes (padding up to the image height) must read as zero
+    for (int i = threadIdx.x; i < q_img_bytes / 16; i += kThreads)
         reinterpret_cast<int4 *>(q_img0)[i] = make_int4(0, 0, 0, 0);
     fence_proxy_async_smem();
     tc_fence_before_sync();
@@ -414,7 +442,7 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     if (warp == 0) {
         // ================================================================== producer
         uint32_t issued = 0;          // key tiles requested so far
-        QState qs = {{-1, -1}, {0, 0}, {0, 0}};
+        QState qs = {-1, 0, 0};
         if (lane == 0) {
             tma_prefetch_desc(&kmap);
             tma_prefetch_desc(&qmap);
@@ -424,23 +452,21 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
             bool ok = true;
             while (ok && next_entry(a, cur, e)) {
                 if (e.n_tiles == 0) continue;
-                const int qb = e.qbuf;
-                if (qs.unit[qb] != e.unit) {
+                if (qs.unit != e.unit) {
                     // the MMAs that read the old image must have completed (signalled by the MMA warp
                     // when it reaches this item)
-                    if (qs.unit[qb] != -1) {
-                        ok = mbar_wait(&bar.qfree[qb], qs.uses[qb] & 1u, &abort_s);
-                        ++qs.uses[qb];
+                    if (qs.unit != -1) {
+                        ok = mbar_wait(&bar.qfree, qs.frees & 1u, &abort_s);
+                        ++qs.frees;
                         if (!ok) break;
                     }
-                    mbar_arrive_expect_tx(&bar.qfull[qb], (uint32_t)(a.q_copies * a.kblocks * s.R * 128));
-                    uint8_t *img = q_img0 + qb * q_img_bytes;
+                    mbar_arrive_expect_tx(&bar.qfull, (uint32_t)(a.q_copies * a.kblocks * s.R * 128));
                     for (int cp = 0; cp < a.q_copies; ++cp)
                         for (int kb = 0; kb < a.kblocks; ++kb)
-                            tma_load_4d(img + kb * kQRegion + cp * a.Rp * 128, &qmap, &bar.qfull[qb], kb * 64, 0,
+                            tma_load_4d(q_img0 + kb * kQRegion + cp * a.Rp * 128, &qmap, &bar.qfull, kb * 64, 0,
                                         e.h * s.G, e.b);
-                    qs.unit[qb] = e.unit;
-                    ++qs.loads[qb];
+                    qs.unit = e.unit;
+                    ++qs.loads;
                 }
                 const int tok0 = (int)e.off + e.j_begin;
                 const int bcoord = s.cu ? 0 : e.b;
@@ -471,11 +497,10 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                     mbar_wait(&bar.full[st], (g / kStages) & 1, &never);
                 }
             }
-            for (int qb = 0; qb < 2; ++qb)
-                if (qs.loads[qb] > 0) {
-                    volatile int never = 0;
-                    mbar_wait(&bar.qfull[qb], (qs.loads[qb] - 1) & 1u, &never);
-                }
+            if (qs.loads > 0) {
+                volatile int never = 0;
+                mbar_wait(&bar.qfull, (qs.loads - 1) & 1u, &never);
+            }
         }
         __syncwarp();
         // the tail of the gather: the idle tile ring becomes copy slots
@@ -490,28 +515,27 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         // ================================================================== MMA issue
         if (lane == 0) {
             uint32_t it = 0;
-            QState qs = {{-1, -1}, {0, 0}, {0, 0}};
+            QState qs = {-1, 0, 0};
             Cursor cur;
             cursor_init(cur);
             Entry e;
+            const uint64_t q_desc0 = umma_desc_sw128(smem_u32(q_img0));
             const uint64_t k_desc0 = umma_desc_sw128(smem_u32(k_stage0));
             const uint32_t stage_step = (uint32_t)stage_bytes >> 4;
             bool ok = true;
             while (ok && next_entry(a, cur, e)) {
                 if (e.n_tiles == 0) continue;
-                const int qb = e.qbuf;
-                if (qs.unit[qb] != e.unit) {
-                    if (qs.unit[qb] != -1) {
-                        umma_commit(&bar.qfree[qb]);      // arrives once every MMA issued so far has completed
-                        ++qs.uses[qb];
+                if (qs.unit != e.unit) {
+                    if (qs.unit != -1) {
+                        umma_commit(&bar.qfree);          // arrives once every MMA issued so far has completed
+                        ++qs.frees;
                     }
-                    ok = mbar_wait(&bar.qfull[qb], qs.loads[qb] & 1u, &abort_s);
-                    ++qs.loads[qb];
-                    qs.unit[qb] = e.unit;
+                    ok = mbar_wait(&bar.qfull, qs.loads & 1u, &abort_s);
+                    ++qs.loads;
+                    qs.unit = e.unit;
                     if (!ok) break;
                     tc_fence_after_sync();
                 }
-                const uint64_t q_desc0 = umma_desc_sw128(smem_u32(q_img0 + qb * q_img_bytes));
                 const bool sweep2 = e.phase != 0;
                 const uint32_t idesc = sweep2 ? umma_idesc_bf16(128, a.r16) : umma_idesc_bf16(128, kTile);
                 for (int t = 0; t < e.n_tiles; ++t) {
@@ -529,11 +553,14 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                     tc_fence_after_sync();
                     const uint64_t k_desc = k_desc0 + (uint64_t)(st * stage_step);
                     const uint32_t d_tmem = tmem_base + buf * 128;
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint32_t qo = (uint32_t)((ks >> 2) * kQRegion + (ks & 3) * 32) >> 4;
-                        const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
-                        if (sweep2) umma_bf16(d_tmem, k_desc + ko, q_desc0 + qo, idesc, ks > 0);
-                        else umma_bf16(d_tmem, q_desc0 + qo, k_desc + ko, idesc, ks > 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        if (ks < ksteps) {
+                            const uint32_t qo = (uint32_t)((ks >> 2) * kQRegion + (ks & 3) * 32) >> 4;
+                            const uint32_t ko = (uint32_t)((ks >> 2) * kRegion + (ks & 3) * 32) >> 4;
+                            if (sweep2) umma_bf16(d_tmem, k_desc + ko, q_desc0 + qo, idesc, ks > 0);
+                            else umma_bf16(d_tmem, q_desc0 + qo, k_desc + ko, idesc, ks > 0);
+                        }
                     }
                     umma_commit(&bar.tfull[buf]);
                     umma_commit(&bar.empty[st]);
@@ -557,11 +584,8 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         while (!aborted && next_entry(a, cur, e)) {
             if (e.phase == 0) {
                 // ---------------------------------------------------------- statistics sweep (Eq. 1)
-                float2 *out = a.stats + ((size_t)e.unit * a.n_stat_chunks + e.chunk) * a.r_pad;
-                if (e.n_tiles == 0) {
-                    for (int r = tl; r < a.r_pad; r += kComputeThreads) out[r] = make_float2(-INFINITY, 0.f);
-                    continue;
-                }
+                unsigned long long *out = a.pstats + ((size_t)e.unit * a.n_stat_chunks + e.chunk) * 128;
+                if (e.n_tiles == 0) continue;        // a chunk without keys: nobody reads its entries
                 {
                     const int col0 = (L / Rp) * Rp;                 // warp-uniform: Rp is a multiple of 32
                     const int nslot = Rp >> 5;                      // 32-column slots this thread reduces
@@ -590,21 +614,19 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                 compute_sync();
                 // combine the compute groups and the column slices of each row, in a fixed order
                 const int copies = 128 / Rp;
-                for (int r = tl; r < a.r_pad; r += kComputeThreads) {
-                    float2 res = make_float2(-INFINITY, 0.f);
-                    if (r < s.R) {
-                        float M = -INFINITY;
-                        for (int g = 0; g < kBufs; ++g)
-                            for (int cp = 0; cp < copies; ++cp) M = fmaxf(M, part[g][r + cp * Rp].x);
-                        float sum = 0.f;
-                        for (int g = 0; g < kBufs; ++g)
-                            for (int cp = 0; cp < copies; ++cp) {
-                                const float2 p = part[g][r + cp * Rp];
-                                if (p.y > 0.f) sum += p.y * fast_exp2((p.x - M) * c);
-                            }
-                        res = make_float2(M * c, sum);
-                    }
-                    out[r] = res;
+                if (tl < s.R) {
+                    const int r = tl;
+                    float M = -INFINITY;
+                    for (int g = 0; g < kBufs; ++g)
+                        for (int cp = 0; cp < copies; ++cp) M = fmaxf(M, part[g][r + cp * Rp].x);
+                    float sum = 0.f;
+                    for (int g = 0; g < kBufs; ++g)
+                        for (int cp = 0; cp < copies; ++cp) {
+                            const float2 p = part[g][r + cp * Rp];
+                            if (p.y > 0.f) sum += p.y * fast_exp2((p.x - M) * c);
+                        }
+                    // published as it is written: no fence, no counter
+                    st_relaxed_gpu_u64(out + r, stat_pack(M * c, sum));
                 }
                 // uniform over the compute warps: nobody leaves the list while others still synchronise
                 int any;
@@ -612,8 +634,6 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                              "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
                              : "=r"(any) : "r"((int)abort_s), "n"(kBarCompute), "n"(kComputeThreads) : "memory");
                 aborted = any;
-                // release: cumulative over what the compute warps wrote before the barrier above
-                if (tl == 0 && !aborted) red_release_gpu_add(a.sync + kSyncTickets + kSyncWordsPerUnit * e.unit + 1, 1);
                 continue;
             }
             // -------------------------------------------------------------- scoring sweep (Eq. 2-4) + selection
@@ -652,20 +672,33 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                 float2 *merged = &part[0][0];
                 const int len1 = tc_chunk_len(e.n, cpu, 1);
                 const int used1 = (e.n + len1 - 1) / len1;   // chunks of the unit that hold keys in the statistics sweep
-                int ok = 1;
-                if (lane == 0) ok = poll_until_at_least(unit_words + 1, used1, &abort_s) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
                 {
                     const int r = tl % 128, mp = tl / 128;
                     float M = -INFINITY, sum = 0.f;
-                    const int used = (r < s.R && ok) ? used1 : 0;
-                    const float2 *st = a.stats + (size_t)e.unit * a.n_stat_chunks * a.r_pad + r;
+                    const int used = r < s.R ? used1 : 0;
+                    const unsigned long long *st = a.pstats + (size_t)e.unit * a.n_stat_chunks * 128 + r;
                     for (int c0 = mp; c0 < used; c0 += 8 * kMergers) {
                         float2 p[8];
+                        // entries that have not been written yet read as zero: look again (bounded)
+                        unsigned long long t0 = 0;
+                        for (uint32_t spin = 1;; ++spin) {
+                            bool all = true;
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const int cidx = c0 + u * kMergers;
-                            p[u] = cidx < used ? __ldcg(st + (size_t)cidx * a.r_pad) : make_float2(-INFINITY, 0.f);
+                            for (int u = 0; u < 8; ++u) {
+                                const int cidx = c0 + u * kMergers;
+                                p[u] = make_float2(-INFINITY, 0.f);
+                                if (cidx < used) all &= stat_unpack(ld_relaxed_gpu_u64(st + (size_t)cidx * 128), p[u]);
+                            }
+                            if (all) break;
+                            if (*static_cast<volatile int *>(&abort_s)) break;
+                            if ((spin & 63u) == 0u) {
+                                const unsigned long long now = global_timer_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > 2 * kWaitLimitNs) {
+                                    abort_s = 1;
+                                    break;
+                                }
+                            }
                         }
                         float Mn = M;
 #pragma unroll
@@ -770,7 +803,7 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                 if (tl == 0) red_release_gpu_add(unit_words, 1);
             } else {
                 if (tl == 0 && poll_until_at_least(unit_words, used2 - 1, &abort_s)) {
-                    atomicExch(unit_words, 0);       // every other block of the unit is past its waits
+                    atomicExch(unit_words, 0);       // every other block of the unit has read what it needs
                     atomicExch(unit_words + 1, 0);
                 }
                 asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
@@ -778,6 +811,13 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                              : "=r"(any) : "r"((int)abort_s), "n"(kBarCompute), "n"(kComputeThreads) : "memory");
                 aborted = any;
                 if (aborted) break;
+                if (!a.lse_obs) {
+                    // the unit's statistics entries go back to "not written" for the next launch
+                    const int len1 = tc_chunk_len(e.n, cpu, 1);
+                    const int used1 = (e.n + len1 - 1) / len1;
+                    unsigned long long *st = a.pstats + (size_t)e.unit * a.n_stat_chunks * 128;
+                    for (int i = tl; i < used1 * 128; i += kComputeThreads) st[i] = 0ull;
+                }
                 if (a.window_idx) {
                     select_topk_block<kComputeThreads, kBarCompute, 64>(
                         topk_sm, a.window_scores + (size_t)e.unit * s.kw_max, kw,
@@ -905,7 +945,7 @@ PipeDevice *pipe_device()
 
 size_t pipe_smem_bytes(int kblocks)
 {
-    return 1024 + (size_t)2 * kblocks * kQRegion + (size_t)kStages * kblocks * kRegion +
+    return 1024 + (size_t)kblocks * kQRegion + (size_t)kStages * kblocks * kRegion +
            (size_t)kCopyWarps * kCopySlots * kCopySlotBytes;
 }
 
@@ -971,7 +1011,7 @@ int launch_group_pipeline(const KShape &ks, const void *q, const void *k, float 
 
     PipeArgs a;
     a.s = ks;
-    a.stats = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + ws.stats_off);
+    a.pstats = reinterpret_cast<unsigned long long *>(static_cast<char *>(workspace) + ws.pstats_off);
     a.window_scores = window_scores;
     a.token_scores = token_scores;
     a.lse_obs = lse_obs;
@@ -980,7 +1020,6 @@ int launch_group_pipeline(const KShape &ks, const void *q, const void *k, float 
     a.status = reinterpret_cast<int *>(static_cast<char *>(workspace) + ws.status_off);
     a.sync = reinterpret_cast<int *>(static_cast<char *>(workspace) + ws.sync_off);
     a.n_stat_chunks = ws.n_stat_chunks;
-    a.r_pad = ws.r_pad;
     const int units = ks.batch * ks.hkv;
     const PipePlan plan = pipe_plan(units, ks.max_seqlen, ks.d);
     a.chunks_per_unit = plan.chunks_per_unit;

@@ -42,6 +42,8 @@ Workspace plan_workspace(const KShape &ks)
     off = 64;
     w.sync_off = off;
     off = align_up(off + (kSyncTickets + kSyncWordsPerUnit * (size_t)units) * sizeof(int), 256);
+    w.pstats_off = off;
+    off = align_up(off + (ks.R <= 128 ? units * w.n_stat_chunks * 128 * sizeof(unsigned long long) : 0), 256);
     w.stats_off = off;
     off = align_up(off + units * w.n_stat_chunks * w.r_pad * sizeof(float2), 256);
     w.lse_off = off;
@@ -86,7 +88,7 @@ int resolve(const wkv_shape *s, KShape &ks)
         set_error_detail("task %d unknown", s->task);
         return WKV_ERR_SHAPE;
     }
-    if (s->score_impl < WKV_SCORE_AUTO || s->score_impl > WKV_SCORE_TCGEN05_UNFUSED || s->reserved != 0) {
+    if (s->score_impl < WKV_SCORE_AUTO || s->score_impl > WKV_SCORE_TCGEN05_PIPELINED || s->reserved != 0) {
         set_error_detail("score_impl %d / reserved %d invalid", s->score_impl, s->reserved);
         return WKV_ERR_SHAPE;
     }
@@ -199,7 +201,7 @@ static int check_workspace(const Workspace &ws, const void *workspace, size_t by
 static int pick_score_impl(const wkv_shape *s, const KShape &ks, const Workspace &ws, bool &use_tc)
 {
     const bool tc_ok = score_tc_supported(ks, s->dtype);
-    if ((s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_UNFUSED) && !tc_ok) {
+    if ((s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_PIPELINED) && !tc_ok) {
         set_error_detail("tensor-core score kernels need bf16, head_dim 64/128 and G*alpha <= 256 on a device of "
                          "compute capability 10");
         return WKV_ERR_UNSUPPORTED;
@@ -229,17 +231,22 @@ int do_score(const wkv_shape *s, const KShape &ks, const Workspace &ws, const vo
     int st = pick_score_impl(s, ks, ws, use_tc);
     if (st != WKV_OK) return st;
     if (use_tc) {
-        const bool forced = s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_UNFUSED;
+        const bool forced = s->score_impl == WKV_SCORE_TCGEN05 || s->score_impl == WKV_SCORE_TCGEN05_PIPELINED;
         st = WKV_ERR_UNSUPPORTED;
-        if (s->score_impl != WKV_SCORE_TCGEN05_UNFUSED && group_pipeline_supported(ks, s->dtype)) {
+        if (s->score_impl == WKV_SCORE_TCGEN05_PIPELINED) {
+            if (!group_pipeline_supported(ks, s->dtype)) {
+                set_error_detail("the pipelined kernel needs G*alpha <= 128 and observation positions as the faster "
+                                 "dimension of Q_obs");
+                return WKV_ERR_UNSUPPORTED;
+            }
             // one launch for scoring, selection and (when asked and possible) the gather
             const bool fuse = gather && window_idx && group_pipeline_can_gather(ks, elem_bytes(s->dtype), gather->n_tensors);
             st = launch_group_pipeline(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws,
                                        stream, lse_obs, fuse ? gather : nullptr);
             if (st == WKV_OK && fuse && gathered) *gathered = true;
+            return st;
         }
-        if (st == WKV_ERR_UNSUPPORTED)
-            st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream,
+        st = launch_score_tc(ks, q, k, window_scores, token_scores, window_idx, kept_len, workspace, ws, stream,
                                  lse_obs);
         // a key layout that no tensor map can describe is served by the CUDA-core kernels
         if (st != WKV_ERR_UNSUPPORTED || forced) return st;

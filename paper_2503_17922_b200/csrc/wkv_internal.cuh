@@ -76,6 +76,8 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
 struct Workspace {
     size_t status_off;   // int: device status word, only ever OR-ed by the kernels (0 = no error)
     size_t sync_off;     // int [kSyncTickets + kSyncWordsPerUnit * units], self-resetting
+    size_t pstats_off;   // u64 [units][n_stat_chunks][128]: self-validating (max, sum) entries of the pipelined kernel;
+                         // zero between launches (the kernel that writes them clears them again)
     size_t stats_off;    // float2 [units][n_stat_chunks][R_pad]  partial (max, sum) per row
     size_t lse_off;      // float  [units][R_pad]                 log2 of the row normaliser
     size_t scores_off;   // float  [units][kw_max]                window scores when the caller passes none

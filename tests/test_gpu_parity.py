@@ -15,13 +15,15 @@ pytestmark = pytest.mark.gpu
 
 # "tc" forces the tensor-core (tcgen05) score kernels, "simt" the CUDA-core ones; the full-size
 # configuration tests below use AUTO, which picks the tensor-core kernels for bf16 inputs
-IMPLS = {"simt": binding.WKV_SCORE_SIMT, "tc": binding.WKV_SCORE_TCGEN05, "auto": binding.WKV_SCORE_AUTO}
+IMPLS = {"simt": binding.WKV_SCORE_SIMT, "tc": binding.WKV_SCORE_TCGEN05, "auto": binding.WKV_SCORE_AUTO,
+         "pipe": binding.WKV_SCORE_TCGEN05_PIPELINED}
 
 
 def impl_for(w, impl):
-    """fp32 inputs have no tensor-core path: forcing it must be refused, so those cases run AUTO."""
-    if impl == "tc" and w.dtype == "f32":
-        prob = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05)
+    """fp32 inputs have no tensor-core path, and the pipelined kernel takes at most 128 observation
+    rows: forcing either must be refused, so those cases run AUTO."""
+    if (impl in ("tc", "pipe") and w.dtype == "f32") or (impl == "pipe" and w.rows > 128):
+        prob = binding.Problem.from_workload(w, score_impl=IMPLS[impl])
         with pytest.raises(binding.WkvError) as e:
             binding.wkv_score_windows(prob, torch.zeros(16, device="cuda"), torch.zeros(16, device="cuda"),
                                       torch.zeros(16, device="cuda"), None, prob.alloc_workspace())
@@ -40,7 +42,7 @@ def small(dtype="bf16", **kw):
 
 
 # ------------------------------------------------------------------ whole path, small shapes
-@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
 @pytest.mark.parametrize("case", [
     dict(),                                                   # bf16, R = 64, ragged last window
     dict(task=wl.TASK_AGGREGATION, top_p=3),
@@ -68,7 +70,7 @@ def test_group_small(case, impl):
 
 
 # ------------------------------------------------------------------ normalisers supplied by the caller
-@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
 @pytest.mark.parametrize("staged", [False, True])
 @pytest.mark.parametrize("case", [
     dict(),
@@ -88,7 +90,7 @@ def test_group_with_given_normalisers(case, staged, impl):
     assert max_rel < 1e-4
 
 
-@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
 @pytest.mark.parametrize("given_lse", [False, True])
 def test_layer_by_layer_use_equals_the_group_call(given_lse, impl):
     """The leader is scored and selected alone, then every layer of the group is gathered by its own
@@ -138,7 +140,7 @@ def test_group_plan_replays_the_group_call():
         before = binding.wkv_launch_count()
         plan.launch()
         torch.cuda.synchronize()
-        assert binding.wkv_launch_count() - before >= 1          # one launch when the pipelined kernel also gathers
+        assert binding.wkv_launch_count() - before >= 2
         assert binding.device_status(work) == 0
         ref = pu.run_gpu_group(w, grp)
         np.testing.assert_array_equal(out["window_idx"].cpu().numpy(), ref["window_idx"])
@@ -158,13 +160,15 @@ def test_group_plan_replays_the_group_call():
                           out["kept_len"], work, keep_capacity=1)          # refused at creation, as by the direct call
 
 
-def test_expired_wait_sets_the_status_word_and_the_context_survives():
-    """Every wait inside the fused kernel is bounded.  Here the arrival count of unit 0 is set so far
-    below zero that it can never reach its target: the blocks of that unit give up after about a
-    second, the kernel ends, bit 0 of the status word is set, and after zeroing the workspace the
-    same call works again.  The arrival word is located through wkv_workspace_sync_words."""
+@pytest.mark.parametrize("impl", ["tc", "pipe"])
+def test_expired_wait_sets_the_status_word_and_the_context_survives(impl):
+    """Every wait inside the fused kernel is bounded.  Here the ticket count of unit 0 is set so far
+    below zero that it can never reach its target: the block that waits for it gives up after about
+    two seconds (and with it every warp waiting for that unit's selection), the kernel ends, bit 0 of
+    the status word is set, and after zeroing the workspace the same call works again.  The word is
+    located through wkv_workspace_sync_words."""
     w = small()
-    prob = binding.Problem.from_workload(w, score_impl=binding.WKV_SCORE_TCGEN05)
+    prob = binding.Problem.from_workload(w, score_impl=IMPLS[impl])
     grp = wl.make_group(w, 0)
     q = binding.to_device(grp["q_obs"])
     ks = [binding.to_device(x) for x in grp["k_layers"]]
@@ -173,13 +177,13 @@ def test_expired_wait_sets_the_status_word_and_the_context_survives():
     work = prob.alloc_workspace()
     ticket_off, arrival_off = binding.workspace_sync_words(prob, 0)
     assert arrival_off == ticket_off + 4 and arrival_off % 4 == 0 and arrival_off < work.numel()
-    work[arrival_off: arrival_off + 4].view(torch.int32)[0] = -1000000
+    work[ticket_off: ticket_off + 4].view(torch.int32)[0] = -1000000
     binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
                                out["kept_len"], work, keep_capacity=out["keep_capacity"])
     torch.cuda.synchronize()                      # returns: nothing hangs
     assert binding.device_status(work) & 1
     work.zero_()
-    gpu = pu.run_gpu_group(w, grp, score_impl=binding.WKV_SCORE_TCGEN05)
+    gpu = pu.run_gpu_group(w, grp, score_impl=IMPLS[impl])
     binding.wkv_compress_group(prob, q, ks, vs, out["k_out"], out["v_out"], out["window_scores"], out["window_idx"],
                                out["kept_len"], work, keep_capacity=out["keep_capacity"])
     torch.cuda.synchronize()
@@ -211,7 +215,7 @@ def test_stage_entry_points_and_token_scores(impl):
     assert rel.max() < 1e-4
 
 
-@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
 def test_token_major_key_layout(impl):
     # K/V stored [B, N, H_kv, d] (head stride < token stride): another order of tensor-map dimensions
     w = small(batch=2, max_seqlen=777, window=16, task=wl.TASK_AGGREGATION, top_p=5)
@@ -473,7 +477,7 @@ def _run_host_entry(w, grp):
                                     out["k_out"], out["v_out"], out["window_idx"], out["kept_len"],
                                     out["keep_capacity"], work)
     # the call returns after synchronising its stream: the host buffers are complete here
-    assert binding.wkv_launch_count() - before >= 1
+    assert binding.wkv_launch_count() - before >= 2
     assert binding.device_status(work) == 0
     return {"prob": prob, "window_idx": h_idx.numpy().copy(), "kept_len": h_kept.numpy().copy(),
             "k_out": [binding.to_host_bits(t) for t in h_k_out], "v_out": [binding.to_host_bits(t) for t in h_v_out],
@@ -505,7 +509,7 @@ def test_launches_are_counted_and_errors_raise():
     w = small()
     before = binding.wkv_launch_count()
     pu.run_gpu_group(w, wl.make_group(w, 0))
-    assert binding.wkv_launch_count() - before >= 1     # one pipelined launch, or score+selection and gather
+    assert binding.wkv_launch_count() - before >= 2     # fused score+selection launch, gather launch
     prob = binding.Problem.from_workload(w)
     with pytest.raises(binding.WkvError):
         binding.wkv_score_windows(prob, None, None, None, None, prob.alloc_workspace())
@@ -541,6 +545,17 @@ def test_config3_with_the_localization_flag():
     w = wl.scaled(wl.llama8b_full(), task=wl.TASK_LOCALIZATION)
     grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=7)
     assert gpu["prob"].k_max == 243 and max_rel < 1e-4
+
+
+@pytest.mark.parametrize("which", ["config2", "config3", "config4"])
+def test_pipelined_single_launch_form_on_full_configs(which):
+    """The opt-in single-launch kernel (statistics sweep one wave ahead, gather by bulk copies inside the
+    launch) on full-size configurations: same bars against the oracle as the default path."""
+    w = {"config2": wl.llama8b_single_group(wl.TASK_AGGREGATION), "config3": wl.llama8b_full(),
+         "config4": wl.mistral_needle(16384, 0.5)}[which]
+    before = binding.wkv_launch_count()
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, group=1 if w.n_groups > 1 else 0, score_impl=IMPLS["pipe"])
+    assert binding.wkv_launch_count() - before == 1 and max_rel < 1e-4
 
 
 def test_config3_with_given_normalisers():
