@@ -136,6 +136,20 @@ int32_t wkv_keep_max(const wkv_shape *s); /* max_b (k_b*omega + min(alpha, n_b))
 int wkv_group_budgets(int32_t n_layers, int32_t gamma, int64_t b_total, int32_t lambda_num, int32_t lambda_den,
                       int32_t *per_layer_out);
 
+/*
+ * Jaccard similarity of retained-window index sets (section 3.2, the intra-group similarity the
+ * index sharing of section 2.2.2 rests on): |A n B| / |A u B| per unit for two selections of the same
+ * batch, e.g. the lists two different layers would select.  Host function on HOST arrays, no device
+ * work.
+ *   idx_a, idx_b   HOST int32 [units, k_max]: ascending window indices, padded with negative entries
+ *                  (the layout wkv_select_topk_windows writes, copied to the host)
+ *   per_unit_out   HOST out or NULL, double [units]; two empty sets count as identical (1.0)
+ *   mean_out       HOST out or NULL: the mean over the units
+ * Returns WKV_ERR_SHAPE for non-positive sizes or a list that is not strictly ascending.
+ */
+int wkv_jaccard_windows(const int32_t *idx_a, const int32_t *idx_b, int32_t units, int32_t k_max,
+                        double *per_unit_out, double *mean_out);
+
 /* Bytes of DEVICE scratch that wkv_score_windows / wkv_compress_group need for this
  * shape (256-byte aligned base expected).  Returns 0 for an invalid shape. */
 size_t wkv_workspace_bytes(const wkv_shape *s);
@@ -230,6 +244,43 @@ int wkv_gather_kv(const wkv_shape *s, int32_t n_layers,
                   const int32_t *window_idx,
                   void *const *k_out_layers, void *const *v_out_layers,
                   const int32_t *cu_seqlens_out, int32_t keep_capacity, void *cuda_stream);
+
+/*
+ * The same gather into a PAGED compact cache (section 2.2.2; the cache that the decode phase of
+ * section 2.1 attends over, in the block-table form serving engines keep it in).  Row r of unit (b, h)
+ * goes to page block_table[b][r / page_size], slot r % page_size; pool element (page, h, slot, c) lives
+ * at  pool[page*page_stride + h*head_stride + slot*row_stride + c]  (e.g. [pages, H_kv, page_size, d]:
+ * page_stride = H_kv*page_size*d, head_stride = page_size*d, row_stride = d; token-major pages
+ * [pages, page_size, H_kv, d]: head_stride = d, row_stride = H_kv*d).  One block table serves every
+ * layer and both K and V, as the index sharing of the group implies; per-unit lengths are kept_len.
+ *   k_pool_layers, v_pool_layers   HOST arrays [n_layers] of DEVICE pool pointers (v may be NULL with v_layers)
+ *   block_table   DEVICE int32 [B, max_pages]; an entry outside [0, num_pages) makes its rows be skipped
+ *   max_pages * page_size must cover wkv_keep_max(); strides in elements, multiples of 16 bytes
+ * Other arguments as wkv_gather_kv.
+ */
+int wkv_gather_kv_paged(const wkv_shape *s, int32_t n_layers,
+                        const void *const *k_layers, const void *const *v_layers,
+                        const int32_t *window_idx,
+                        void *const *k_pool_layers, void *const *v_pool_layers,
+                        const int32_t *block_table, int32_t max_pages, int32_t page_size, int32_t num_pages,
+                        int64_t page_stride, int64_t head_stride, int64_t row_stride, void *cuda_stream);
+
+/*
+ * Compaction in place (section 2.2.2 as it is driven during prefill: a layer's compact cache takes the
+ * place of its full K/V).  For every layer tensor and every unit, the retained rows (selected windows
+ * in ascending position, then the observation rows) are moved to the front of the unit's own rows,
+ * in the tensor's own layout: afterwards row r < kept_len of unit (b, h) holds what wkv_gather_kv would
+ * have written to row r of the compact cache; rows from kept_len on hold leftovers.  Rows only move
+ * toward lower addresses; the kernel orders the reads of a stretch of rows before the writes that land
+ * on them (one thread block walks a unit's rows in ascending batches), so the result is exact.
+ *   k_layers, v_layers   HOST arrays [n_layers] of DEVICE pointers, read AND written (v_layers may be NULL)
+ *   window_idx           DEVICE int32 [B, H_kv, wkv_k_max()], an ascending selection as written by
+ *                        wkv_select_topk_windows; entries that are no window of the sequence or lie
+ *                        before their own slot are skipped (their rows stay as they are)
+ * A row of head_dim elements may be at most 128 KB.
+ */
+int wkv_compact_kv_inplace(const wkv_shape *s, int32_t n_layers, void *const *k_layers, void *const *v_layers,
+                           const int32_t *window_idx, void *cuda_stream);
 
 /*
  * One layer group (sections 2.2.1-2.2.2): score + select on k_layers[0] with q_obs_leader,

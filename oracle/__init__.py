@@ -11,6 +11,7 @@ paper's steps on numpy arrays:
   select_leader       Eq. 1-4 + selection for every unit of a batch
   gather_layer        compacted cache of one layer from shared indices
   compress_group      the whole group (leader selection + gamma gathers)
+  jaccard_windows     similarity of two index selections (section 3.2)
 
 bf16 tensors are passed as uint16 bit patterns, fp32 as float32.
 """
@@ -223,6 +224,20 @@ def group_budgets(n_layers: int, gamma: int, b_total: int, lam) -> Dict[str, obj
     ints = [int(x // 1) for x in per_layer]
     ints[0] += (b_total - gamma * sum(ints)) // gamma
     return {"group": b, "per_layer": per_layer, "per_layer_int": ints}
+
+
+def jaccard_windows(idx_a: np.ndarray, idx_b: np.ndarray) -> np.ndarray:
+    """Section 3.2: Jaccard similarity |A n B| / |A u B| of two retained-window sets per unit, written
+    out with Python sets.  idx_* are [..., k_max] index lists padded with negative entries; two empty
+    sets count as identical."""
+    a = np.asarray(idx_a)
+    b = np.asarray(idx_b)
+    out = np.zeros(a.shape[:-1], dtype=np.float64)
+    for pos in np.ndindex(*a.shape[:-1]):
+        A = {int(x) for x in a[pos] if x >= 0}
+        B = {int(x) for x in b[pos] if x >= 0}
+        out[pos] = 1.0 if not (A | B) else len(A & B) / len(A | B)
+    return out
 
 
 def keep_max(seqlens: Sequence[int], budgets: Sequence[int], l_obs: int, window: int) -> int:

@@ -22,8 +22,8 @@ WKV_SCORE_AUTO, WKV_SCORE_SIMT, WKV_SCORE_TCGEN05, WKV_SCORE_TCGEN05_PIPELINED =
 WKV_MAX_GROUP_LAYERS = 32
 
 EXPORTED_SYMBOLS = [
-    "wkv_num_windows", "wkv_num_selected", "wkv_keep_len", "wkv_workspace_sync_words", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets",
-    "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv",
+    "wkv_num_windows", "wkv_num_selected", "wkv_keep_len", "wkv_workspace_sync_words", "wkv_kw_max", "wkv_k_max", "wkv_keep_max", "wkv_group_budgets", "wkv_jaccard_windows",
+    "wkv_workspace_bytes", "wkv_score_windows", "wkv_score_windows_static", "wkv_select_topk_windows", "wkv_gather_kv", "wkv_gather_kv_paged", "wkv_compact_kv_inplace",
     "wkv_compress_group", "wkv_compress_group_host", "wkv_score_windows_lse", "wkv_compress_group_lse",
     "wkv_select_leader_windows", "wkv_probe_ex2_rate", "wkv_probe_colsum_rate", "wkv_group_plan_create", "wkv_group_plan_launch", "wkv_group_plan_destroy", "wkv_status_string", "wkv_last_error_detail",
     "wkv_launch_count",
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         getattr(L, name).argtypes = [sp]
     L.wkv_group_budgets.restype = ctypes.c_int
     L.wkv_group_budgets.argtypes = [i32, i32, ctypes.c_int64, i32, i32, vp]
+    L.wkv_jaccard_windows.restype = ctypes.c_int
+    L.wkv_jaccard_windows.argtypes = [vp, vp, i32, i32, vp, ctypes.POINTER(ctypes.c_double)]
     L.wkv_workspace_bytes.restype = sz
     L.wkv_workspace_bytes.argtypes = [sp]
     L.wkv_score_windows.restype = ctypes.c_int
@@ -103,6 +105,11 @@ def lib() -> ctypes.CDLL:
     L.wkv_select_topk_windows.argtypes = [sp, vp, vp, vp, vp]
     L.wkv_gather_kv.restype = ctypes.c_int
     L.wkv_gather_kv.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
+    L.wkv_gather_kv_paged.restype = ctypes.c_int
+    L.wkv_gather_kv_paged.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, i32, i32, i32, ctypes.c_int64, ctypes.c_int64,
+                                      ctypes.c_int64, vp]
+    L.wkv_compact_kv_inplace.restype = ctypes.c_int
+    L.wkv_compact_kv_inplace.argtypes = [sp, i32, vp, vp, vp, vp]
     L.wkv_compress_group.restype = ctypes.c_int
     L.wkv_compress_group.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     L.wkv_score_windows_lse.restype = ctypes.c_int
@@ -287,6 +294,22 @@ def wkv_gather_kv(prob: Problem, k_layers, v_layers, window_idx, k_out_layers, v
                                _ptr_array(v_layers), _ptr(window_idx), _ptr_array(k_out_layers),
                                _ptr_array(v_out_layers), _ptr(cu_seqlens_out), keep_capacity, _stream(stream)),
            "wkv_gather_kv")
+
+
+def wkv_gather_kv_paged(prob: Problem, k_layers, v_layers, window_idx, k_pools, v_pools, block_table, page_size: int,
+                        num_pages: int, page_stride: int, head_stride: int, row_stride: int, stream=None) -> None:
+    """Gather into paged pools: row r of unit (b, h) -> page block_table[b, r // page_size], slot r % page_size."""
+    _check(lib().wkv_gather_kv_paged(ctypes.byref(prob.shape), len(k_layers), _ptr_array(k_layers), _ptr_array(v_layers),
+                                     _ptr(window_idx), _ptr_array(k_pools), _ptr_array(v_pools), _ptr(block_table),
+                                     block_table.shape[-1], page_size, num_pages, page_stride, head_stride, row_stride,
+                                     _stream(stream)), "wkv_gather_kv_paged")
+
+
+def wkv_compact_kv_inplace(prob: Problem, k_layers, v_layers, window_idx, stream=None) -> None:
+    """Moves every unit's retained rows to the front of its own rows, inside the given tensors."""
+    _check(lib().wkv_compact_kv_inplace(ctypes.byref(prob.shape), len(k_layers), _ptr_array(k_layers),
+                                        _ptr_array(v_layers), _ptr(window_idx), _stream(stream)),
+           "wkv_compact_kv_inplace")
 
 
 def wkv_compress_group(prob: Problem, q_obs_leader, k_layers, v_layers, k_out_layers, v_out_layers,
@@ -494,6 +517,21 @@ def wkv_group_budgets(n_layers: int, gamma: int, b_total: int, lambda_num: int =
     _check(lib().wkv_group_budgets(n_layers, gamma, b_total, lambda_num, lambda_den, out.ctypes.data),
            "wkv_group_budgets")
     return out
+
+
+def wkv_jaccard_windows(idx_a: np.ndarray, idx_b: np.ndarray):
+    """Section 3.2's similarity of two selections: (per-unit Jaccard [units], mean).  Host arrays
+    [..., k_max] of ascending window indices padded with negative entries."""
+    a = np.ascontiguousarray(idx_a, dtype=np.int32)
+    b = np.ascontiguousarray(idx_b, dtype=np.int32)
+    assert a.shape == b.shape
+    k_max = a.shape[-1]
+    units = a.size // k_max
+    per_unit = np.zeros(units, dtype=np.float64)
+    mean = ctypes.c_double(0.0)
+    _check(lib().wkv_jaccard_windows(a.ctypes.data, b.ctypes.data, units, k_max, per_unit.ctypes.data,
+                                     ctypes.byref(mean)), "wkv_jaccard_windows")
+    return per_unit.reshape(a.shape[:-1]), float(mean.value)
 
 
 def wkv_launch_count() -> int:

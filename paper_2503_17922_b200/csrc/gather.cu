@@ -26,6 +26,10 @@ struct GatherParams {
     int elem_bytes;
     int slots_per_block;              // windows (selected + observation) handled by one block
     int obs_slots;                    // ceil(alpha / omega)
+    // paged output (page_size > 0): row r of unit (b, h) lives in page block_table[b][r / page_size]
+    const int *block_table;           // [batch][max_pages]
+    int max_pages, page_size, num_pages;
+    long long page_vecs, head_vecs, row_vecs;   // strides of the page pool in 16-byte vectors
 };
 
 __device__ __forceinline__ int4 ld_stream(const int4 *p)
@@ -79,7 +83,10 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
         dst = reinterpret_cast<int4 *>(prm.tab.dst[tensor]) + (long long)unit * prm.keep_capacity * vpr;
         dst_row_vecs = vpr;
     }
-    const bool src_dense = src_row_vecs == vpr, dst_dense = dst_row_vecs == vpr;
+    const bool paged = prm.page_size > 0;
+    const bool src_dense = src_row_vecs == vpr, dst_dense = dst_row_vecs == vpr && !paged;
+    const int *pages = paged ? prm.block_table + (size_t)b * prm.max_pages : nullptr;
+    if (paged) dst = reinterpret_cast<int4 *>(prm.tab.dst[tensor]) + (long long)h * prm.head_vecs;
 
     const int slot_end = min(k + prm.obs_slots, (int)(blockIdx.x + 1) * prm.slots_per_block);
     for (int slot = blockIdx.x * prm.slots_per_block + warp; slot < slot_end; slot += kWarps) {
@@ -101,7 +108,33 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
         if (n_rows <= 0) continue;
         // dense output: a unit owns keep_capacity rows (cannot trigger while the device copies of
         // cu_seqlens / budgets equal the host copies the capacity was checked against)
-        if (!prm.cu_out && dst_row0 + n_rows > prm.keep_capacity) continue;
+        if (!prm.cu_out && !paged && dst_row0 + n_rows > prm.keep_capacity) continue;
+        if (paged) {
+            // every row finds its page; a row whose page entry is missing or negative is skipped
+            const int n_vec = n_rows * vpr;
+            for (int v0 = lane; v0 < n_vec; v0 += 32 * kBatch) {
+                int4 val[kBatch];
+                long long doff[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int v = v0 + u * 32;
+                    doff[u] = -1;
+                    if (v < n_vec) {
+                        const int r = prm.vec_shift >= 0 ? v >> prm.vec_shift : v / vpr;
+                        const int c = v - r * vpr;
+                        const int row = dst_row0 + r, page = row / prm.page_size;
+                        const int phys = page < prm.max_pages ? pages[page] : -1;
+                        if (phys >= 0 && phys < prm.num_pages)
+                            doff[u] = (long long)phys * prm.page_vecs + (long long)(row - page * prm.page_size) * prm.row_vecs + c;
+                        val[u] = ld_stream(src + (long long)(src_row0 + r) * src_row_vecs + c);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    if (doff[u] >= 0) st_stream(dst + doff[u], val[u]);
+            }
+            continue;
+        }
         const int4 *sp = src + src_row0 * src_row_vecs;
         int4 *dp = dst + dst_row0 * dst_row_vecs;
         const int n_vec = n_rows * vpr;
@@ -134,9 +167,21 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
 
 cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const LayerTable &tab,
                           const int *window_idx, const int *cu_out, int keep_capacity,
-                          cudaStream_t stream)
+                          cudaStream_t stream, const PagedOut *paged)
 {
     GatherParams prm;
+    prm.block_table = nullptr;
+    prm.max_pages = prm.page_size = prm.num_pages = 0;
+    prm.page_vecs = prm.head_vecs = prm.row_vecs = 0;
+    if (paged) {
+        prm.block_table = paged->block_table;
+        prm.max_pages = paged->max_pages;
+        prm.page_size = paged->page_size;
+        prm.num_pages = paged->num_pages;
+        prm.page_vecs = paged->page_stride * elem_bytes / 16;
+        prm.head_vecs = paged->head_stride * elem_bytes / 16;
+        prm.row_vecs = paged->row_stride * elem_bytes / 16;
+    }
     prm.s = ks;
     prm.tab = tab;
     prm.window_idx = window_idx;

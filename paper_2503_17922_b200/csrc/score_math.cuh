@@ -128,5 +128,53 @@ __device__ __forceinline__ float pool_window_sorted(const float *w, int size, in
     return acc / (float)p_eff;
 }
 
+// Eq. 4 for one window of 64 or 128 tokens by one warp: lane l holds elements l, l + 32, ... in
+// registers; a bitonic sorting network over (register, lane) orders them descending (partners 32 or
+// more apart are registers of the same lane, closer ones are exchanged by shuffle), then the p largest
+// are summed: per lane in ascending rank, across lanes by a fixed butterfly, so the result is the same
+// from run to run.  Positions beyond `size` hold -inf.  Every lane returns the window score.
+template <int omega>
+__device__ __forceinline__ float pool_window_warp(const float *w, int size, int p, int lane)
+{
+    constexpr int NR = omega / 32;
+    static_assert(omega == 64 || omega == 128, "window length");
+    float v[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) v[r] = r * 32 + lane < size ? w[r * 32 + lane] : -INFINITY;
+#pragma unroll
+    for (int k = 2; k <= omega; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            if (j >= 32) {
+                const int jj = j >> 5;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    if ((r & jj) == 0) {
+                        const float hi = fmaxf(v[r], v[r | jj]), lo = fminf(v[r], v[r | jj]);
+                        const bool descending = ((r * 32 + lane) & k) == 0;
+                        v[r] = descending ? hi : lo;
+                        v[r | jj] = descending ? lo : hi;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const float other = __shfl_xor_sync(0xffffffffu, v[r], j);
+                    const bool lower = (lane & j) == 0;
+                    const bool descending = ((r * 32 + lane) & k) == 0;
+                    v[r] = (lower == descending) ? fmaxf(v[r], other) : fminf(v[r], other);
+                }
+            }
+        }
+    }
+    const int p_eff = p < size ? p : size;
+    float acc = 0.f;
+#pragma unroll
+    for (int r = 0; r < NR; ++r) acc += (r * 32 + lane < p_eff) ? v[r] : 0.f;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc / (float)p_eff;
+}
+
 }  // namespace
 }  // namespace wkv

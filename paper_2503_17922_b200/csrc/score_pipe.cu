@@ -781,6 +781,14 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                         else r = pool_window_sorted<4>(t_chunk + lo, size, s.p);
                         ws_out[i] = r;
                     }
+                } else if (s.omega == 64 || s.omega == 128) {
+                    // one warp per window
+                    for (int lw = tl >> 5; lw < n_win; lw += kComputeWarps) {
+                        const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
+                        const float r = s.omega == 64 ? pool_window_warp<64>(t_chunk + lo, size, s.p, lane)
+                                                      : pool_window_warp<128>(t_chunk + lo, size, s.p, lane);
+                        if (lane == 0) ws_out[lw] = r;
+                    }
                 } else {
                     for (int lw = tl; lw < n_win; lw += kComputeThreads) {
                         const int lo = lw * s.omega;

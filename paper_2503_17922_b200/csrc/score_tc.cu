@@ -613,6 +613,15 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
                         ws_out[lw] = r;
                     }
                 }
+                else if (s.omega == 64 || s.omega == 128) {
+                    // one warp per window
+                    for (int lw = warp; lw < n_win; lw += kThreads / 32) {
+                        const int lo = lw * s.omega, size = min(s.omega, n_tok - lo);
+                        const float r = s.omega == 64 ? pool_window_warp<64>(t_item + lo, size, s.p, lane)
+                                                      : pool_window_warp<128>(t_item + lo, size, s.p, lane);
+                        if (lane == 0) ws_out[lw] = r;
+                    }
+                }
                 else {
                     for (int lw = threadIdx.x; lw < n_win; lw += kThreads) {
                         const int lo = lw * s.omega;

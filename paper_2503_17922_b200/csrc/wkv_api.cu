@@ -404,6 +404,55 @@ int wkv_group_budgets(int32_t n_layers, int32_t gamma, int64_t b_total, int32_t 
     return WKV_OK;
 }
 
+int wkv_jaccard_windows(const int32_t *idx_a, const int32_t *idx_b, int32_t units, int32_t k_max,
+                        double *per_unit_out, double *mean_out)
+{
+    if (!idx_a || !idx_b) {
+        set_error_detail("idx_a / idx_b is NULL");
+        return WKV_ERR_NULL;
+    }
+    if (units < 1 || k_max < 1) {
+        set_error_detail("jaccard: units %d, k_max %d", units, k_max);
+        return WKV_ERR_SHAPE;
+    }
+    double total = 0.0;
+    for (int u = 0; u < units; ++u) {
+        const int32_t *a = idx_a + (size_t)u * k_max, *b = idx_b + (size_t)u * k_max;
+        int na = 0, nb = 0;
+        while (na < k_max && a[na] >= 0) ++na;
+        while (nb < k_max && b[nb] >= 0) ++nb;
+        for (int i = 1; i < na; ++i)
+            if (a[i] <= a[i - 1]) {
+                set_error_detail("jaccard: list A of unit %d is not strictly ascending at entry %d", u, i);
+                return WKV_ERR_SHAPE;
+            }
+        for (int i = 1; i < nb; ++i)
+            if (b[i] <= b[i - 1]) {
+                set_error_detail("jaccard: list B of unit %d is not strictly ascending at entry %d", u, i);
+                return WKV_ERR_SHAPE;
+            }
+        // merge walk over two ascending lists
+        int i = 0, j = 0, both = 0;
+        while (i < na && j < nb) {
+            if (a[i] == b[j]) {
+                ++both;
+                ++i;
+                ++j;
+            } else if (a[i] < b[j]) {
+                ++i;
+            } else {
+                ++j;
+            }
+        }
+        const int either = na + nb - both;
+        const double jac = either == 0 ? 1.0 : (double)both / (double)either;
+        if (per_unit_out) per_unit_out[u] = jac;
+        total += jac;
+    }
+    if (mean_out) *mean_out = total / units;
+    return WKV_OK;
+}
+
 size_t wkv_workspace_bytes(const wkv_shape *s)
 {
     KShape ks;
@@ -505,6 +554,96 @@ int wkv_gather_kv(const wkv_shape *s, int32_t n_layers, const void *const *k_lay
     return check_cuda(launch_gather(ks, elem_bytes(s->dtype), n_tensors, tab, window_idx, cu_seqlens_out,
                                     keep_capacity, static_cast<cudaStream_t>(cuda_stream)),
                       "gather kernel");
+}
+
+int wkv_gather_kv_paged(const wkv_shape *s, int32_t n_layers, const void *const *k_layers,
+                        const void *const *v_layers, const int32_t *window_idx, void *const *k_pool_layers,
+                        void *const *v_pool_layers, const int32_t *block_table, int32_t max_pages,
+                        int32_t page_size, int32_t num_pages, int64_t page_stride, int64_t head_stride,
+                        int64_t row_stride, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!window_idx || !block_table) {
+        set_error_detail("window_idx / block_table is NULL");
+        return WKV_ERR_NULL;
+    }
+    LayerTable tab;
+    int n_tensors = 0;
+    st = fill_table(n_layers, k_layers, v_layers, k_pool_layers, v_pool_layers, tab, n_tensors);
+    if (st != WKV_OK) return st;
+    const int eb = elem_bytes(s->dtype);
+    if (max_pages < 1 || page_size < 1 || num_pages < 1 || (long long)max_pages * page_size < keep_max_of(s)) {
+        set_error_detail("paged cache: max_pages %d x page_size %d does not cover the %d rows a unit may keep "
+                         "(num_pages %d)", max_pages, page_size, keep_max_of(s), num_pages);
+        return WKV_ERR_SHAPE;
+    }
+    const int64_t strides[3] = {page_stride, head_stride, row_stride};
+    for (int i = 0; i < 3; ++i)
+        if (strides[i] < 0 || (strides[i] * eb) % 16) {
+            set_error_detail("paged cache: stride #%d = %lld is negative or not 16-byte aligned", i, (long long)strides[i]);
+            return WKV_ERR_ALIGN;
+        }
+    if (row_stride < s->head_dim) {
+        set_error_detail("paged cache: row stride smaller than head_dim");
+        return WKV_ERR_SHAPE;
+    }
+    PagedOut po;
+    po.block_table = block_table;
+    po.max_pages = max_pages;
+    po.page_size = page_size;
+    po.num_pages = num_pages;
+    po.page_stride = page_stride;
+    po.head_stride = head_stride;
+    po.row_stride = row_stride;
+    return check_cuda(launch_gather(ks, eb, n_tensors, tab, window_idx, nullptr, 0,
+                                    static_cast<cudaStream_t>(cuda_stream), &po),
+                      "gather kernel (paged output)");
+}
+
+int wkv_compact_kv_inplace(const wkv_shape *s, int32_t n_layers, void *const *k_layers, void *const *v_layers,
+                           const int32_t *window_idx, void *cuda_stream)
+{
+    KShape ks;
+    int st = resolve(s, ks);
+    if (st != WKV_OK) return st;
+    if (!window_idx || !k_layers) {
+        set_error_detail("window_idx / k_layers is NULL");
+        return WKV_ERR_NULL;
+    }
+    if (n_layers < 1 || n_layers > WKV_MAX_GROUP_LAYERS) {
+        set_error_detail("n_layers %d outside 1..%d", n_layers, WKV_MAX_GROUP_LAYERS);
+        return WKV_ERR_LIMIT;
+    }
+    const int eb = elem_bytes(s->dtype);
+    if ((long long)s->head_dim * eb > 128 * 1024) {
+        set_error_detail("in-place compaction: a row of %lld bytes exceeds 128 KB", (long long)s->head_dim * eb);
+        return WKV_ERR_UNSUPPORTED;
+    }
+    InplaceTable tab;
+    int n_tensors = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        void *p[2] = {k_layers[l], v_layers ? v_layers[l] : nullptr};
+        for (int t = 0; t < (v_layers ? 2 : 1); ++t) {
+            if (!p[t]) {
+                set_error_detail("layer %d: NULL tensor pointer", l);
+                return WKV_ERR_NULL;
+            }
+            if (!aligned16(p[t])) {
+                set_error_detail("layer %d: tensor pointer not 16-byte aligned", l);
+                return WKV_ERR_ALIGN;
+            }
+            for (int o = 0; o < n_tensors; ++o)
+                if (tab.ptr[o] == p[t]) {
+                    set_error_detail("layer %d: the same tensor is listed twice", l);
+                    return WKV_ERR_SHAPE;
+                }
+            tab.ptr[n_tensors++] = p[t];
+        }
+    }
+    return check_cuda(launch_compact_inplace(ks, eb, n_tensors, tab, window_idx, static_cast<cudaStream_t>(cuda_stream)),
+                      "in-place compaction kernel");
 }
 
 }  // extern "C"

@@ -206,9 +206,21 @@ struct LayerTable {
     const void *src[2 * WKV_MAX_GROUP_LAYERS];
     void *dst[2 * WKV_MAX_GROUP_LAYERS];
 };
+// paged compact cache: strides of the page pool in elements
+struct PagedOut {
+    const int *block_table;   // device [batch][max_pages]
+    int max_pages, page_size, num_pages;
+    long long page_stride, head_stride, row_stride;
+};
 cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const LayerTable &tab,
                           const int *window_idx, const int *cu_out, int keep_capacity,
-                          cudaStream_t stream);
+                          cudaStream_t stream, const PagedOut *paged = nullptr);
+// compaction of every layer's K/V inside its own buffer (compact.cu)
+struct InplaceTable {
+    void *ptr[2 * WKV_MAX_GROUP_LAYERS];
+};
+cudaError_t launch_compact_inplace(const KShape &ks, int elem_bytes, int n_tensors, const InplaceTable &tab,
+                                   const int *window_idx, cudaStream_t stream);
 
 // Eq. 4 for one window of `size` values: mean of the p largest.  Elements are visited in the
 // strict order (value descending, position ascending), so equal values are each taken once.

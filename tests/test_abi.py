@@ -166,6 +166,34 @@ def test_gather_refuses_a_cache_that_is_its_own_input(L):
     assert b"must not be the input" in L.wkv_last_error_detail()
 
 
+def test_jaccard_of_index_sets(L):
+    """Section 3.2's similarity measure: closed cases (identical, disjoint, nested, both empty), and the
+    library's merge walk against the oracle's set arithmetic on random selections."""
+    pad = lambda xs, k: np.array(list(xs) + [-1] * (k - len(xs)), dtype=np.int32)
+    a = np.stack([pad([0, 3, 5, 9], 6), pad([1, 2], 6), pad([0, 1, 2, 3], 6), pad([], 6), pad([4], 6)])
+    b = np.stack([pad([0, 3, 5, 9], 6), pad([3, 4], 6), pad([1, 2], 6), pad([], 6), pad([], 6)])
+    per_unit, mean = binding.wkv_jaccard_windows(a, b)
+    assert per_unit.tolist() == [1.0, 0.0, 0.5, 1.0, 0.0] and abs(mean - 0.5) < 1e-15
+    np.testing.assert_array_equal(per_unit, oracle.jaccard_windows(a, b))
+    g = np.random.Generator(np.random.Philox(key=5))
+    A = np.full((3, 4, 40), -1, dtype=np.int32)
+    B = np.full((3, 4, 40), -1, dtype=np.int32)
+    for pos in np.ndindex(3, 4):
+        for M in (A, B):
+            n = int(g.integers(0, 41))
+            M[pos][:n] = np.sort(g.choice(100, size=n, replace=False))
+    per_unit, mean = binding.wkv_jaccard_windows(A, B)
+    ref = oracle.jaccard_windows(A, B)
+    np.testing.assert_allclose(per_unit, ref, rtol=0, atol=1e-15)
+    assert abs(mean - ref.mean()) < 1e-12
+    # symmetric, and 1 only for equal sets
+    np.testing.assert_array_equal(per_unit, binding.wkv_jaccard_windows(B, A)[0])
+    bad = a.copy()
+    bad[0, :2] = [3, 3]
+    with pytest.raises(binding.WkvError):
+        binding.wkv_jaccard_windows(bad, b)
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libwkv.so")

@@ -69,6 +69,22 @@ def test_group_small(case, impl):
                 assert set(planted) <= set(gpu["window_idx"][b, h, :k].tolist())
 
 
+# ------------------------------------------------------------------ the paper's wide review windows (window-size sweep up to 128)
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
+@pytest.mark.parametrize("omega", [64, 128])
+@pytest.mark.parametrize("p_of", ["1", "half", "omega-1", "omega"])
+def test_wide_windows(omega, p_of, impl):
+    """Review windows of 64 and 128 tokens, pooled by one warp per window with a sorting network:
+    p = 1 (max pooling), omega / 2, omega - 1 and omega (mean pooling), with a ragged last window
+    (3,571 review tokens) and a last chunk that holds a partial window."""
+    p = {"1": 1, "half": omega // 2, "omega-1": omega - 1, "omega": omega}[p_of]
+    task = wl.TASK_LOCALIZATION if p == omega else wl.TASK_AGGREGATION
+    w = small(window=omega, task=task, top_p=p, max_seqlen=3587, l_obs=16, budget_frac=0.35, n_planted=3)
+    grp, ref, gpu, (max_rel, swaps) = pu.full_check(w, score_impl=impl_for(w, impl))
+    assert max_rel < 1e-4
+    assert gpu["prob"].kw_max == -(-(3587 - 16) // omega)
+
+
 # ------------------------------------------------------------------ normalisers supplied by the caller
 @pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
 @pytest.mark.parametrize("staged", [False, True])
