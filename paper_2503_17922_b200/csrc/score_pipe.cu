@@ -218,8 +218,8 @@ __device__ __forceinline__ bool next_entry(const PipeArgs &a, Cursor &c, Entry &
                 e.b = e.unit / s.hkv;
                 e.h = e.unit % s.hkv;
                 if (s.cu) {
-                    const int lo = s.cu[e.b];
-                    e.n = min(max(s.cu[e.b + 1] - lo, 0), s.n_cap);
+                    const int lo = min(max(s.cu[e.b], 0), s.total_rows);
+                    e.n = min(min(max(s.cu[e.b + 1] - s.cu[e.b], 0), s.n_cap), s.total_rows - lo);
                     e.off = lo;
                 } else {
                     e.n = s.max_seqlen;

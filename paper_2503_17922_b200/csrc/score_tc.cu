@@ -203,8 +203,8 @@ score_windows_tc(const __grid_constant__ CUtensorMap tmap, const __grid_constant
         im.b = unit / s.hkv;
         im.h = unit % s.hkv;
         if (s.cu) {
-            const int lo = s.cu[im.b];
-            im.n = min(max(s.cu[im.b + 1] - lo, 0), s.n_cap);
+            const int lo = min(max(s.cu[im.b], 0), s.total_rows);
+            im.n = min(min(max(s.cu[im.b + 1] - s.cu[im.b], 0), s.n_cap), s.total_rows - lo);
             im.off = lo;
         } else {
             im.n = s.max_seqlen;

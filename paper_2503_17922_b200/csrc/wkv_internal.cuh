@@ -62,7 +62,10 @@ __device__ inline SeqInfo seq_info(const KShape &s, int b)
     if (s.cu) {
         int lo = s.cu[b];
         r.n = s.cu[b + 1] - lo;
+        // a device copy that disagrees with the host copy must not lead outside the packed tensor
+        lo = lo < 0 ? 0 : (lo > s.total_rows ? s.total_rows : lo);
         r.n = r.n < 0 ? 0 : (r.n > s.n_cap ? s.n_cap : r.n);
+        if (r.n > s.total_rows - lo) r.n = s.total_rows - lo;
         r.off = lo;
     } else {
         r.n = s.max_seqlen;

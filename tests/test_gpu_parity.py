@@ -521,6 +521,45 @@ def test_host_buffer_entry_point(which):
             np.testing.assert_array_equal(got["v_out"][layer], ref["v_out"][layer])
 
 
+@pytest.mark.parametrize("impl", ["simt", "tc", "pipe"])
+def test_stale_device_copy_of_cu_seqlens_stays_in_bounds(impl):
+    """cu_seqlens and budgets exist as a host and a device copy, and sizes are derived from the host
+    one.  If the device copy disagrees (here: other split points, a first sequence longer than any the
+    host copy knows, and an end beyond the packed tensor), results are wrong, but no kernel may touch
+    memory outside the arrays that were sized from the host copy: guard bands around every output
+    keep their pattern, and the call completes without a device error."""
+    w = small(ragged=True, batch=3, max_seqlen=700, n_planted=0)
+    grp = wl.make_group(w, 0)
+    prob = binding.Problem.from_workload(w, score_impl=IMPLS[impl])
+    stale = prob.cu_host.copy()
+    stale[1] += 150                          # sequence 0 longer than max_seqlen allows, sequence 1 shorter
+    stale[-1] += 4000                        # the last sequence would run past the packed tensor
+    prob.cu_dev.copy_(torch.from_numpy(stale))
+    prob.budgets_dev.fill_(10 ** 6)          # and a budget that asks for every window
+    q = binding.to_device(grp["q_obs"])
+    ks = [binding.to_device(x) for x in grp["k_layers"]]
+    vs = [binding.to_device(x) for x in grp["v_layers"]]
+    G = 4096                                 # guard elements on both sides of every output
+
+    def guarded(n, dtype, fill):
+        t = torch.full((n + 2 * G,), fill, dtype=dtype, device="cuda")
+        return t, t[G:G + n]
+    units = w.batch * w.n_kv_heads
+    cap = prob.keep_max
+    bufs = {"scores": guarded(units * prob.kw_max, torch.float32, 7.0),
+            "idx": guarded(units * prob.k_max, torch.int32, -7),
+            "kept": guarded(units, torch.int32, -7)}
+    outs = [guarded(units * cap * w.head_dim, torch.bfloat16, 3.0) for _ in range(2 * w.gamma)]
+    work = prob.alloc_workspace()
+    binding.wkv_compress_group(prob, q, ks, vs, [o[1] for o in outs[: w.gamma]], [o[1] for o in outs[w.gamma:]],
+                               bufs["scores"][1], bufs["idx"][1], bufs["kept"][1], work, keep_capacity=cap)
+    torch.cuda.synchronize()                 # no fault, no hang
+    assert binding.device_status(work) == 0
+    for name, (full, inner) in list(bufs.items()) + [(f"out{i}", o) for i, o in enumerate(outs)]:
+        fill = full[0].item()
+        assert (full[:G] == fill).all() and (full[-G:] == fill).all(), f"{name}: a guard band was written"
+
+
 def test_launches_are_counted_and_errors_raise():
     w = small()
     before = binding.wkv_launch_count()
