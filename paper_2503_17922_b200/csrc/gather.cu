@@ -47,6 +47,9 @@ __device__ __forceinline__ void st_stream(int4 *p, const int4 &v)
                  : "memory");
 }
 
+// PAGED is a separate instantiation: its per-row page arithmetic would otherwise cost the plain copy
+// registers it needs for its loads in flight.
+template <bool PAGED>
 __global__ void __launch_bounds__(kThreads, 4)
 gather_kv_kernel(const __grid_constant__ GatherParams prm)
 {
@@ -83,7 +86,7 @@ gather_kv_kernel(const __grid_constant__ GatherParams prm)
         dst = reinterpret_cast<int4 *>(prm.tab.dst[tensor]) + (long long)unit * prm.keep_capacity * vpr;
         dst_row_vecs = vpr;
     }
-    const bool paged = prm.page_size > 0;
+    constexpr bool paged = PAGED;
     const bool src_dense = src_row_vecs == vpr, dst_dense = dst_row_vecs == vpr && !paged;
     const int *pages = paged ? prm.block_table + (size_t)b * prm.max_pages : nullptr;
     if (paged) dst = reinterpret_cast<int4 *>(prm.tab.dst[tensor]) + (long long)h * prm.head_vecs;
@@ -200,7 +203,8 @@ cudaError_t launch_gather(const KShape &ks, int elem_bytes, int n_tensors, const
     prm.slots_per_block = (int)per_block;
     const int max_slots = ks.k_max + prm.obs_slots;
     dim3 grid((max_slots + prm.slots_per_block - 1) / prm.slots_per_block, ks.batch * ks.hkv, n_tensors);
-    gather_kv_kernel<<<grid, kThreads, 0, stream>>>(prm);
+    if (paged) gather_kv_kernel<true><<<grid, kThreads, 0, stream>>>(prm);
+    else gather_kv_kernel<false><<<grid, kThreads, 0, stream>>>(prm);
     count_launches(1);
     return cudaGetLastError();
 }

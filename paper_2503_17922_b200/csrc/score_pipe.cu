@@ -691,6 +691,7 @@ group_pipeline_tc(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                             }
                             if (all) break;
                             if (*static_cast<volatile int *>(&abort_s)) break;
+                            __nanosleep(100);     // 512 threads look again: leave the L2 to the blocks still publishing
                             if ((spin & 63u) == 0u) {
                                 const unsigned long long now = global_timer_ns();
                                 if (t0 == 0) t0 = now;

@@ -123,7 +123,7 @@ __host__ __device__ inline TcPlan tc_plan(int units, int max_seqlen, int head_di
     const int max_tiles = (max_seqlen + kTcTileKeys - 1) / kTcTileKeys;
     // A unit needs at least ceil(max_tiles / kTcMaxChunkTiles) blocks: no more units in a wave than
     // the SMs can take at that rate, or some blocks get two items of a wave and the others wait for
-    // them (8 sequences of up to 64 K keys: 0.70 ms with 4 units of 37 chunks per wave, 1.18 ms with 5 units of 32).
+    // them.
     const int min_chunks = (max_tiles + kTcMaxChunkTiles - 1) / kTcMaxChunkTiles;
     if (upw > kTcTargetBlocks / min_chunks) upw = kTcTargetBlocks / min_chunks;
     if (upw < 1) upw = 1;
