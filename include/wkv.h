@@ -366,7 +366,11 @@ void wkv_group_plan_destroy(wkv_group_plan *plan);
  * The same group with every tensor in HOST memory (pinned memory recommended): the
  * inputs are copied to caller-provided DEVICE staging buffers, the group is
  * compressed there, and indices, kept lengths and the compact caches are copied
- * back; the function returns after the stream has been synchronised.
+ * back; the function returns after everything it enqueued has completed.  The copies
+ * dominate, so the call runs as a pipeline over the layers: the leader's keys first
+ * (scored and selected as soon as they have landed), then layer by layer copy in, gather,
+ * and copy back on a second stream of the call's own, so that both copy directions are
+ * busy at once.  (This creates and destroys one stream and one event per call.)
  *   *_host arguments    HOST pointers / HOST arrays of HOST pointers
  *   *_dev arguments     DEVICE staging of the same sizes (HOST arrays of DEVICE pointers)
  *   bytes_per_layer     size of one K (or V) tensor; out_bytes_per_layer of one compact cache

@@ -771,34 +771,51 @@ int wkv_compress_group_host(const wkv_shape *s, int32_t n_layers, const void *q_
         }
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    st = check_cuda(cudaMemcpyAsync(q_obs_dev, q_obs_host, q_bytes, cudaMemcpyHostToDevice, stream), "copy of q_obs");
-    for (int l = 0; l < n_layers && st == WKV_OK; ++l) {
-        st = check_cuda(cudaMemcpyAsync(k_layers_dev[l], k_layers_host[l], bytes_per_layer,
-                                        cudaMemcpyHostToDevice, stream), "copy of K");
-        if (st == WKV_OK)
-            st = check_cuda(cudaMemcpyAsync(v_layers_dev[l], v_layers_host[l], bytes_per_layer,
-                                            cudaMemcpyHostToDevice, stream), "copy of V");
-    }
+    // The copies in dominate this call, so it is laid out as a pipeline over the layers: the leader's
+    // keys go first and are scored as soon as they have landed; every layer is gathered behind its own
+    // copy in, and its compact cache travels back on a second stream while the next layer is still
+    // coming in (the two copy directions run at the same time).
+    cudaStream_t back = nullptr;
+    cudaEvent_t ready = nullptr;
+    st = check_cuda(cudaStreamCreateWithFlags(&back, cudaStreamNonBlocking), "stream for the copies back");
     if (st != WKV_OK) return st;
-    st = wkv_compress_group(s, n_layers, q_obs_dev, k_layers_dev, v_layers_dev, k_out_layers_dev,
-                            v_out_layers_dev, nullptr, window_idx_dev, kept_len_dev, nullptr, keep_capacity,
-                            workspace, workspace_bytes, cuda_stream);
-    if (st != WKV_OK) return st;
+    st = check_cuda(cudaEventCreateWithFlags(&ready, cudaEventDisableTiming), "event");
     const size_t units = (size_t)ks.batch * ks.hkv;
-    st = check_cuda(cudaMemcpyAsync(window_idx_host, window_idx_dev, units * ks.k_max * sizeof(int32_t),
-                                    cudaMemcpyDeviceToHost, stream), "copy of window_idx");
+    auto h2d = [&](void *dst, const void *src, size_t bytes, const char *what) {
+        if (st == WKV_OK) st = check_cuda(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream), what);
+    };
+    auto d2h_after = [&](void *dst, const void *src, size_t bytes, const char *what) {
+        if (st == WKV_OK) st = check_cuda(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, back), what);
+    };
+    auto hand_over = [&]() {     // what `stream` has done so far precedes what `back` does next
+        if (st == WKV_OK) st = check_cuda(cudaEventRecord(ready, stream), "event record");
+        if (st == WKV_OK) st = check_cuda(cudaStreamWaitEvent(back, ready, 0), "event wait");
+    };
+    h2d(q_obs_dev, q_obs_host, q_bytes, "copy of q_obs");
+    h2d(k_layers_dev[0], k_layers_host[0], bytes_per_layer, "copy of K");
     if (st == WKV_OK)
-        st = check_cuda(cudaMemcpyAsync(kept_len_host, kept_len_dev, units * sizeof(int32_t),
-                                        cudaMemcpyDeviceToHost, stream), "copy of kept_len");
+        st = wkv_select_leader_windows(s, q_obs_dev, k_layers_dev[0], nullptr, nullptr, window_idx_dev, kept_len_dev,
+                                       workspace, workspace_bytes, cuda_stream);
+    hand_over();
+    d2h_after(window_idx_host, window_idx_dev, units * ks.k_max * sizeof(int32_t), "copy of window_idx");
+    d2h_after(kept_len_host, kept_len_dev, units * sizeof(int32_t), "copy of kept_len");
     for (int l = 0; l < n_layers && st == WKV_OK; ++l) {
-        st = check_cuda(cudaMemcpyAsync(k_out_layers_host[l], k_out_layers_dev[l], out_bytes_per_layer,
-                                        cudaMemcpyDeviceToHost, stream), "copy of compact K");
+        if (l > 0) h2d(k_layers_dev[l], k_layers_host[l], bytes_per_layer, "copy of K");
+        h2d(v_layers_dev[l], v_layers_host[l], bytes_per_layer, "copy of V");
         if (st == WKV_OK)
-            st = check_cuda(cudaMemcpyAsync(v_out_layers_host[l], v_out_layers_dev[l], out_bytes_per_layer,
-                                            cudaMemcpyDeviceToHost, stream), "copy of compact V");
+            st = wkv_gather_kv(s, 1, k_layers_dev + l, v_layers_dev + l, window_idx_dev, k_out_layers_dev + l,
+                               v_out_layers_dev + l, nullptr, keep_capacity, cuda_stream);
+        hand_over();
+        d2h_after(k_out_layers_host[l], k_out_layers_dev[l], out_bytes_per_layer, "copy of compact K");
+        d2h_after(v_out_layers_host[l], v_out_layers_dev[l], out_bytes_per_layer, "copy of compact V");
     }
+    // both streams are drained before the call returns, whatever happened above
+    const cudaError_t e1 = cudaStreamSynchronize(stream), e2 = cudaStreamSynchronize(back);
+    if (ready) cudaEventDestroy(ready);
+    cudaStreamDestroy(back);
     if (st != WKV_OK) return st;
-    return check_cuda(cudaStreamSynchronize(stream), "stream synchronisation");
+    if (e1 != cudaSuccess) return check_cuda(e1, "stream synchronisation");
+    return check_cuda(e2, "stream synchronisation (copies back)");
 }
 
 const char *wkv_status_string(int status)
