@@ -34,6 +34,8 @@ def pick_workload(name: str):
         return wl.llama8b_single_group(wl.TASK_AGGREGATION)
     if name == "C4":
         return wl.mistral_needle(32768, 0.5)
+    if name == "C5-small":
+        return wl.batched_ragged_small()
     return wl.ALL_CONFIGS[name]()
 
 
@@ -247,7 +249,7 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=40)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
+    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5", "C5-small"])
     ap.add_argument("--score-impl", default="auto", choices=["auto", "simt", "tcgen05", "pipelined"])
     ap.add_argument("--groups", type=int, default=0, help="distinct groups kept on the device (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

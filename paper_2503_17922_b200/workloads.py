@@ -143,6 +143,12 @@ def batched_ragged() -> Workload:
                     TASK_AGGREGATION, 16, budget_frac=0.12, ragged=True, n_planted=-1)
 
 
+def batched_ragged_small() -> Workload:
+    """Config 5's shape (256 observation rows per unit, packed ragged batch, 8 layers per group) cut down
+    to 4 sequences of 8-16 K tokens and one group: a case small enough for counter captures."""
+    return scaled(batched_ragged(), name="C5-small", batch=4, max_seqlen=16384, n_layers=8, config_id=13)
+
+
 def qwen_small(l_obs: int = 16, n: int = 8192) -> Workload:
     """The paper's second model family (section 4.1: 7 layers per group, review window 32,
     observation window 4 or 16), with the shape of a 1.5 B model of that family: 28 layers,
