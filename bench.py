@@ -89,15 +89,18 @@ def score_other_floors(w, pk, ex2_per_s: float) -> dict:
             "tensor_floor_ms": flops / (pk["bf16_tflops"] * 1e12) * 1e3}
 
 
+KERNEL_SOURCES = ("score_tc.cu", "score_math.cuh", "tc_common.cuh", "topk_block.cuh", "wkv_internal.cuh", "gather.cu")
+
+
 def kernel_source_hash() -> str:
-    """Fingerprint of the kernel sources: the ncu traffic figures are only quoted while it is unchanged."""
+    """Fingerprint of the sources of the two kernels of the default path (score + selection, gather): the
+    ncu traffic figures are only quoted while it is unchanged."""
     import hashlib
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2503_17922_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
-        if name.endswith((".cu", ".cuh")):
-            h.update(name.encode())
-            h.update(open(os.path.join(csrc, name), "rb").read())
+    for name in KERNEL_SOURCES:
+        h.update(name.encode())
+        h.update(open(os.path.join(csrc, name), "rb").read())
     return h.hexdigest()[:16]
 
 
