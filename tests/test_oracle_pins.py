@@ -307,6 +307,37 @@ def test_gather_into_the_packed_output_layout(ragged):
     assert (out[~written] == FILL).all() and (~written).sum() > 0
 
 
+@pytest.mark.parametrize("ragged", [False, True])
+def test_batch_driver_maps_heads_and_sequences_as_the_library_softmax_does(ragged):
+    """The batch driver (`select_leader`) has to pick, for unit (b, h), sequence b's rows of the packed or
+    dense K, KV head h's keys, and the query heads h*G .. h*G+G-1 (grouped-query attention).  Pinned
+    against an independent library computation per unit: torch CPU softmax with a causal mask, summed
+    over exactly those rows, then average / max pooling by torch for the window scores.  A wrong head
+    mapping, sequence offset or stride gives other scores."""
+    w = wl.scaled(_small_group(ragged=ragged), n_q_heads=6, n_kv_heads=3, task=wl.TASK_LOCALIZATION)
+    grp = wl.make_group(w, 0)
+    res = oracle.select_leader(grp["q_obs"], grp["k_layers"][0], n_kv_heads=w.n_kv_heads, l_obs=w.l_obs,
+                               window=w.window, task=w.task, top_p=w.top_p, max_seqlen=w.max_seqlen,
+                               budgets=grp["budgets"], cu_seqlens=grp["cu_seqlens"], want_tokens=True)
+    q = torch.from_numpy(wl.to_f32(grp["q_obs"])).double()            # [B, H_q, alpha, d]
+    k = torch.from_numpy(wl.to_f32(grp["k_layers"][0])).double()
+    G, a = w.n_q_heads // w.n_kv_heads, w.l_obs
+    for b in range(w.batch):
+        n = int(grp["seqlens"][b])
+        for h in range(w.n_kv_heads):
+            kb = k[int(grp["cu_seqlens"][b]): int(grp["cu_seqlens"][b]) + n, h] if ragged else k[b, h, :n]
+            t = torch.zeros(n - a, dtype=torch.float64)
+            for g in range(G):
+                logits = q[b, h * G + g] @ kb.T / w.head_dim ** 0.5                       # [alpha, n]
+                pos = torch.arange(n - a, n).view(a, 1)
+                logits = logits.masked_fill(torch.arange(n).view(1, n) > pos, float("-inf"))
+                t += torch.softmax(logits, dim=-1)[:, : n - a].sum(0)
+            np.testing.assert_allclose(res["token_scores"][b, h, : n - a], t.numpy(), rtol=1e-10, atol=0)
+            full = (n - a) // w.window
+            pooled = torch.nn.functional.avg_pool1d(t.view(1, 1, -1), w.window, w.window).view(-1).numpy()
+            np.testing.assert_allclose(res["window_scores_f64"][b, h, :full], pooled[:full], rtol=1e-10, atol=0)
+
+
 def test_budget_above_context_is_identity_copy():
     w = wl.scaled(_small_group(), budget_frac=None, budget_tokens=10 ** 6)
     grp = wl.make_group(w, 0)
