@@ -450,6 +450,9 @@ def main() -> None:
                          for d, l in zip(dev_groups, lse)]
             ms_given_lse = time_stage(lse_calls)
     clocks = sampler.stop() if sampler else None
+    if clocks and clocks.get("sm_mhz"):
+        # the step in SM clock cycles: comparable between runs that saw different clocks
+        clocks["sm_cycles_per_step"] = ms_per_step * 1e-3 * clocks["sm_mhz"] * 1e6
 
     pk = peaks()
     floors = score_other_floors(w, pk, ex2_per_s)
